@@ -1,0 +1,244 @@
+// CPU oracle for the error-compensated Gaussian_k sparsifier and exact Top_k.
+//
+// THIS IS TEST INFRASTRUCTURE.  It is a plain, slow, single-threaded
+// restatement of what the paper defines, used only to check the CUDA library
+// and to serve as a timed CPU baseline.  It shares no code with the CUDA path
+// and nothing in the product may call it.
+//
+// Every function names the passage of the paper (arXiv 1911.08772) it follows.
+// Scalars are fp64; the vectors are fp32 because the paper computes in fp32
+// (Section 4.1).  Built with -O2 and without -ffast-math so that signed zeros
+// and denormals survive.
+//
+// Readings taken where the paper is silent (all listed again in the design
+// notes of the repository):
+//   * "std" is the sample standard deviation (divide by d-1).
+//   * ppf(u, p, mu, sigma) is the normal quantile mu + sigma * Phi^-1(p).
+//   * the loop "i = 0 -> 3" runs at most four rounds.
+//   * 2k/3 and 4k/3 are real numbers: tested as 3*est < 2*k and 3*est > 4*k.
+//   * the returned mask is the one last evaluated, i.e. the threshold before
+//     the last adjustment.
+//   * the comparison |u_i| > thres is taken in fp64 (u_i widened exactly).
+//   * k >= d (p <= 0): every element is selected, no statistics.
+//   * exact Top_k breaks ties of equal magnitude toward the lower index.
+//
+// Pins (tests that do not pass through this file's own formulas): see
+// tests/test_oracle_pins.py.  Nothing here is "parity unpinned".
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+extern "C" {
+
+struct oracle_stats {
+    double mu;          // mean of u                          (Alg. 1, statistics)
+    double sigma;       // sample standard deviation of u     (Alg. 1, statistics)
+    double z;           // Phi^-1(1 - k/d)                    (Alg. 1, p and ppf)
+    double thres0;      // mu + sigma * z                     (Alg. 1, ppf)
+    double thr_final;   // threshold of the last evaluated mask
+    int64_t counts[4];  // estimated_k of each executed round (Alg. 1, loop)
+    int32_t rounds;     // rounds executed (1..4), 0 when k >= d
+    int32_t pad;
+    int64_t nnz;        // number of selected elements
+};
+
+// ---------------------------------------------------------------------------
+// Eq. 2: u = g + eps, one IEEE fp32 addition per element.
+// ---------------------------------------------------------------------------
+void oracle_accumulate(const float* g, const float* eps, int64_t d, float* u) {
+    for (int64_t i = 0; i < d; ++i) {
+        u[i] = g[i] + eps[i];
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Alg. 1, "mean and std of vector u": two passes in fp64.
+// unbiased != 0 divides the squared deviations by d-1, otherwise by d.
+// ---------------------------------------------------------------------------
+void oracle_mean_std(const float* u, int64_t d, int unbiased, double* mu, double* sigma) {
+    double s = 0.0;
+    for (int64_t i = 0; i < d; ++i) s += (double)u[i];
+    const double m = s / (double)d;
+    double q = 0.0;
+    for (int64_t i = 0; i < d; ++i) {
+        const double dev = (double)u[i] - m;
+        q += dev * dev;
+    }
+    const double den = unbiased ? (double)(d - 1) : (double)d;
+    *mu = m;
+    *sigma = std::sqrt(q / den);
+}
+
+// ---------------------------------------------------------------------------
+// Standard normal CDF and its inverse (the "ppf" of Alg. 1).
+// Phi(z) = erfc(-z / sqrt 2) / 2.  The inverse is found by bisection on z
+// until the bracket cannot shrink; no coefficient tables.
+// ---------------------------------------------------------------------------
+double oracle_norm_cdf(double z) { return 0.5 * std::erfc(-z / std::sqrt(2.0)); }
+
+double oracle_norm_ppf(double p) {
+    if (!(p > 0.0)) return -std::numeric_limits<double>::infinity();
+    if (!(p < 1.0)) return std::numeric_limits<double>::infinity();
+    double lo = -40.0, hi = 40.0;
+    for (int it = 0; it < 200; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (mid <= lo || mid >= hi) break;
+        if (oracle_norm_cdf(mid) < p) lo = mid; else hi = mid;
+    }
+    // lo and hi are now adjacent doubles; return the one whose CDF is nearer p
+    return (p - oracle_norm_cdf(lo) <= oracle_norm_cdf(hi) - p) ? lo : hi;
+}
+
+// ---------------------------------------------------------------------------
+// Alg. 1, loop body, for one threshold: the mask |u_i| > thres and its number
+// of True values.
+// ---------------------------------------------------------------------------
+int64_t oracle_count_above(const float* u, int64_t d, double thres) {
+    int64_t c = 0;
+    for (int64_t i = 0; i < d; ++i)
+        if ((double)std::fabs(u[i]) > thres) ++c;
+    return c;
+}
+
+// ---------------------------------------------------------------------------
+// Alg. 1 up to the end of its loop: statistics, initial threshold, and the
+// count-and-adjust rounds.
+// Fills st (everything except nnz is final on return; nnz = last count).
+// ---------------------------------------------------------------------------
+void oracle_gaussiank_threshold(const float* u, int64_t d, int64_t k, int max_rounds,
+                                int unbiased, oracle_stats* st) {
+    std::memset(st, 0, sizeof(*st));
+    if (k >= d) {  // p = 1 - k/d <= 0: the quantile is -inf, every element passes
+        st->mu = st->sigma = std::numeric_limits<double>::quiet_NaN();
+        st->z = st->thres0 = st->thr_final = -std::numeric_limits<double>::infinity();
+        st->rounds = 0;
+        st->nnz = d;
+        return;
+    }
+    oracle_mean_std(u, d, unbiased, &st->mu, &st->sigma);       // mu, sigma
+    const double p = 1.0 - (double)k / (double)d;               // p = 1 - k/d
+    st->z = oracle_norm_ppf(p);
+    double thres = st->mu + st->sigma * st->z;                  // ppf(p; mu, sigma)
+    st->thres0 = thres;
+    if (max_rounds > 4) max_rounds = 4;
+    for (int i = 0; i < max_rounds; ++i) {                      // i = 0 .. 3
+        const int64_t est = oracle_count_above(u, d, thres);    // estimated_k
+        st->counts[i] = est;
+        st->rounds = i + 1;
+        st->thr_final = thres;  // the mask of this round is the last one evaluated
+        st->nnz = est;
+        if (3 * est < 2 * k) thres = 0.5 * thres;               // est < 2k/3
+        else if (3 * est > 4 * k) thres = 1.5 * thres;          // est > 4k/3
+        else break;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Alg. 1, final masked assignment, with the compact output form of Section 1 ("with
+// corresponding indices"): pairs (i, u_i) with |u_i| > thres, ascending i.
+// Returns the number of pairs; writes at most cap of them.
+// ---------------------------------------------------------------------------
+int64_t oracle_select(const float* u, int64_t d, double thres, int64_t cap,
+                      int32_t* idx, float* val) {
+    int64_t n = 0;
+    for (int64_t i = 0; i < d; ++i) {
+        if ((double)std::fabs(u[i]) > thres) {
+            if (n < cap) { idx[n] = (int32_t)i; val[n] = u[i]; }
+            ++n;
+        }
+    }
+    return n;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 2: eps_new = u - Comp(u).  Selected slots hold u_i - u_i = +0, the
+// others u_i - 0 = u_i.  idx lists the selected positions.
+// ---------------------------------------------------------------------------
+void oracle_residual(const float* u, int64_t d, const int32_t* idx, const float* val,
+                     int64_t nnz, float* eps_new) {
+    std::vector<float> comp((size_t)d, 0.0f);
+    for (int64_t j = 0; j < nnz; ++j) comp[(size_t)idx[j]] = val[j];
+    for (int64_t i = 0; i < d; ++i) {
+        eps_new[i] = u[i] - comp[(size_t)i];
+    }
+}
+
+// ---------------------------------------------------------------------------
+// One whole sparsifier step (Eq. 2 with Comp = Gaussian_k, Alg. 1).
+// eps is updated in place.  Pairs beyond cap are not emitted and their slots
+// keep u in eps_new, so that Comp(u) + eps_new == u still holds.
+// ---------------------------------------------------------------------------
+int64_t oracle_gk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int64_t cap,
+                           int32_t* idx, float* val, oracle_stats* st) {
+    std::vector<float> u((size_t)d);
+    oracle_accumulate(g, eps, d, u.data());
+    oracle_gaussiank_threshold(u.data(), d, k, 4, 1, st);
+    int64_t n = oracle_select(u.data(), d, st->thr_final, cap, idx, val);
+    if (n > cap) n = cap;
+    oracle_residual(u.data(), d, idx, val, n, eps);
+    return n;
+}
+
+// ---------------------------------------------------------------------------
+// Layer-wise variant: Alg. 1 run independently on each contiguous segment
+// [off[s], off[s+1]) with its own k_s.  Indices are global, segments are
+// emitted in order.  (The paper states Alg. 1 for the whole vector; the
+// segmented form is this repository's workload definition.)
+// ---------------------------------------------------------------------------
+int64_t oracle_gk_sparsify_segmented(const float* g, float* eps, int64_t d,
+                                     const int64_t* off, const int64_t* seg_k, int32_t S,
+                                     int64_t cap, int32_t* idx, float* val,
+                                     int64_t* seg_nnz, oracle_stats* st /* S entries */) {
+    int64_t total = 0;
+    for (int32_t s = 0; s < S; ++s) {
+        const int64_t lo = off[s], n = off[s + 1] - off[s];
+        if (n <= 0) { std::memset(&st[s], 0, sizeof(oracle_stats)); seg_nnz[s] = 0; continue; }
+        const int64_t room = cap > total ? cap - total : 0;
+        const int64_t m = oracle_gk_sparsify(g + lo, eps + lo, n, seg_k[s], room,
+                                             idx + total, val + total, &st[s]);
+        for (int64_t j = 0; j < m; ++j) idx[total + j] += (int32_t)lo;
+        seg_nnz[s] = m;
+        total += m;
+    }
+    (void)d;
+    return total;
+}
+
+// ---------------------------------------------------------------------------
+// Section 1, definition of Top_k: the k entries of largest absolute value with
+// their indices.  Full sort of all d positions by (|u_i| descending, i
+// ascending); the first k are kept and re-emitted in ascending index order.
+// Magnitudes are compared through their IEEE bit patterns with the sign bit
+// cleared, which orders finite non-negative floats exactly as their values
+// (so +0 and -0 tie).
+// ---------------------------------------------------------------------------
+void oracle_topk_exact(const float* u, int64_t d, int64_t k, int32_t* idx, float* val) {
+    std::vector<uint64_t> key((size_t)d);
+    for (int64_t i = 0; i < d; ++i) {
+        uint32_t b;
+        std::memcpy(&b, &u[i], 4);
+        b &= 0x7fffffffu;
+        // larger magnitude first, then lower index first
+        key[(size_t)i] = ((uint64_t)(0x7fffffffu - b) << 32) | (uint64_t)(uint32_t)i;
+    }
+    std::sort(key.begin(), key.end());
+    std::vector<int32_t> chosen((size_t)k);
+    for (int64_t j = 0; j < k; ++j) chosen[(size_t)j] = (int32_t)(key[(size_t)j] & 0xffffffffu);
+    std::sort(chosen.begin(), chosen.end());
+    for (int64_t j = 0; j < k; ++j) { idx[j] = chosen[(size_t)j]; val[j] = u[chosen[(size_t)j]]; }
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 5: ||u - Top_k(u)||^2 / ||u||^2 from the list of kept positions.
+// ---------------------------------------------------------------------------
+double oracle_error_ratio(const float* u, int64_t d, const int32_t* idx, int64_t nnz) {
+    double all = 0.0, kept = 0.0;
+    for (int64_t i = 0; i < d; ++i) all += (double)u[i] * (double)u[i];
+    for (int64_t j = 0; j < nnz; ++j) kept += (double)u[idx[j]] * (double)u[idx[j]];
+    return (all - kept) / all;
+}
+
+}  // extern "C"
