@@ -1,0 +1,182 @@
+/*
+ * gk.h -- C ABI of the B200 error-compensated Gaussian_k gradient sparsifier
+ *         and exact Top_k selection (arXiv 1911.08772).
+ *
+ * Conventions for every call
+ *   - Pointers marked DEVICE are caller-owned global memory of the CUDA device
+ *     that is current when the call is made; pointers marked HOST are ordinary
+ *     host memory.  The library never frees or keeps caller pointers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  All device work is enqueued on it and the call returns without
+ *     synchronising, unless stated otherwise.
+ *   - Vectors are fp32, indices int32, so 1 <= d <= 2^31 - 1.  Base pointers of
+ *     g, eps and u must be 16-byte aligned.  Inputs must be finite.
+ *   - The library owns a small scratch workspace per (device, stream), created
+ *     by the first call that needs it (cudaMalloc; use gk_reserve to do that
+ *     ahead of time).  Two calls that overlap on the GPU must use different
+ *     streams.
+ *   - Return value: GK_OK or a negative gk_status for errors detected on the
+ *     host before anything is enqueued.  Conditions found on the device
+ *     (truncated output, a bounded wait that ran out, a malformed segment
+ *     table) are reported in gk_stats.status, never by a trap or a hang.
+ */
+#ifndef GK_H_
+#define GK_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* gk_stream_t; /* a cudaStream_t */
+
+typedef enum gk_status {
+    GK_OK = 0,
+    GK_ERR_NULL = -1,      /* a required pointer is NULL */
+    GK_ERR_SIZE = -2,      /* d < 1 or d > 2^31 - 1, or S < 1 */
+    GK_ERR_K = -3,         /* k < 1 or k > d */
+    GK_ERR_ALIGN = -4,     /* g / eps / u not 16-byte aligned */
+    GK_ERR_ALIAS = -5,     /* g overlaps eps */
+    GK_ERR_CUDA = -6,      /* a CUDA runtime call failed (see gk_last_cuda_error) */
+    GK_ERR_NOMEM = -7,     /* workspace allocation failed */
+    GK_ERR_CAPACITY = -8,  /* gk_set_capacity: cap < 0 */
+    GK_ERR_LIMIT = -9      /* size beyond a fixed built-in limit */
+} gk_status;
+
+/* Values of gk_stats.status (bit flags, written by the device). */
+#define GK_DEV_OK 0
+#define GK_DEV_TRUNCATED 1    /* more survivors than the output capacity */
+#define GK_DEV_TIMEOUT 2      /* a bounded look-back wait gave up; outputs invalid */
+#define GK_DEV_BAD_SEGMENTS 4 /* seg_offsets not ascending from 0 to d, or seg_k out of range */
+
+/*
+ * What one Gaussian_k run decided (Algorithm 1 of the paper).  For the
+ * segmented call there is one record per segment.
+ */
+typedef struct gk_stats {
+    double mu;         /* mean of u */
+    double sigma;      /* sample standard deviation of u (divisor d - 1) */
+    double z;          /* Phi^-1(1 - k/d) */
+    double thres0;     /* mu + sigma * z, the first threshold */
+    double thr_final;  /* threshold of the mask that was returned */
+    int64_t counts[4]; /* #{|u_i| > thres} seen in each executed round */
+    int32_t rounds;    /* rounds executed, 0 when k >= d (everything selected) */
+    int32_t status;    /* GK_DEV_* flags */
+    int64_t nnz;       /* size of the returned mask (before any truncation) */
+    int64_t emitted;   /* pairs actually written (= min(nnz, capacity)) */
+} gk_stats;
+
+/*
+ * gk_sparsify -- one step of error-compensated sparsification, Eq. 2 of the
+ * paper with Comp_k = Gaussian_k (Algorithm 1):
+ *     u = g + eps;   (idx, val) = Gaussian_k(u);   eps <- u - Comp(u).
+ * Gaussian_k takes mean and standard deviation of u, sets the first threshold
+ * to the normal quantile at p = 1 - k/d, then for at most four rounds counts
+ * #{|u_i| > thres} and halves the threshold when the count is below 2k/3,
+ * multiplies it by 1.5 when above 4k/3, and stops otherwise.  The mask of the
+ * last round evaluated is returned.
+ *
+ *   g        DEVICE in   d floats, the stochastic gradient; must not overlap eps
+ *   eps      DEVICE i/o  d floats; in: residual eps_t, out: eps_{t+1}
+ *                        (+0.0f at selected positions, u_i elsewhere)
+ *   d, k     sizes, 1 <= k <= d
+ *   idx_out  DEVICE out  capacity ints (see gk_set_capacity; default d):
+ *                        positions with |u_i| > threshold, ascending
+ *   val_out  DEVICE out  capacity floats: u at those positions
+ *   nnz_out  DEVICE out  one int64: number of pairs written
+ *   stream   the stream to enqueue on
+ *
+ * The number of survivors is data dependent and may be below or above k
+ * (Appendix A.5 of the paper).  If it exceeds the capacity, only the first
+ * `capacity` survivors in index order are written and only their eps slots are
+ * cleared, so that Comp(u) + eps_{t+1} == u still holds; status gets
+ * GK_DEV_TRUNCATED.
+ */
+int gk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
+/*
+ * gk_sparsify_segmented -- the same step with Algorithm 1 run independently on
+ * every contiguous segment [seg_offsets[s], seg_offsets[s+1]) with its own
+ * mean, deviation, k_s and threshold (layer-wise selection).  The paper states
+ * Algorithm 1 for the whole vector; applying it per layer is this library's
+ * extension.  All S segments are processed by one batched launch per stage.
+ *
+ *   seg_offsets DEVICE in  S + 1 int64, seg_offsets[0] = 0 <= ... <= seg_offsets[S] = d;
+ *                          boundaries need no alignment; empty segments allowed
+ *   seg_k       DEVICE in  S int64, 1 <= seg_k[s] (values >= the segment length
+ *                          select the whole segment)
+ *   S           number of segments, 1 <= S <= 65536
+ *   idx_out / val_out      as above; indices are global, segments appear in order,
+ *                          so idx_out is ascending overall
+ *   seg_nnz_out DEVICE out S int64: size of each segment's mask (may be NULL)
+ *   nnz_out     DEVICE out one int64: total pairs written
+ * A malformed table sets GK_DEV_BAD_SEGMENTS; nothing is then selected
+ * (eps still receives u).
+ */
+int gk_sparsify_segmented(const float* g, float* eps, int64_t d, const int64_t* seg_offsets,
+                          const int64_t* seg_k, int32_t S, int32_t* idx_out, float* val_out,
+                          int64_t* seg_nnz_out, int64_t* nnz_out, gk_stream_t stream);
+
+/*
+ * topk_exact -- Top_k of Section 1 of the paper: the k entries of largest
+ * absolute value with their indices, by radix select on the magnitude bits.
+ * Entries of equal magnitude are taken in order of increasing index (+0 and
+ * -0 tie).  Exactly k pairs are written, in ascending index order.
+ *
+ *   u        DEVICE in   d floats, not modified
+ *   idx_out  DEVICE out  k ints;   val_out  DEVICE out  k floats
+ */
+int topk_exact(const float* u, int64_t d, int64_t k, int32_t* idx_out, float* val_out,
+               gk_stream_t stream);
+
+/*
+ * topk_sparsify -- Eq. 2 of the paper with Comp_k = Top_k: u = g + eps, the exact
+ * Top_k of u is written as k pairs, eps <- u - Top_k(u).  Arguments as for
+ * gk_sparsify; exactly k pairs are written and *nnz_out = k.
+ */
+int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                  float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
+/*
+ * gk_sparsify_host -- gk_sparsify for HOST buffers (Eq. 2, Algorithm 1): copies g
+ * and eps to library-owned device staging buffers, runs the step, copies
+ * eps_{t+1}, the pairs and their count back, and synchronises before
+ * returning.  All pointers are HOST memory (pinned memory makes the copies
+ * faster); idx_out / val_out hold `capacity` entries (default d).
+ */
+int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                     float* val_out, int64_t* nnz_out, gk_stats* stats_out);
+
+/* Output capacity of idx_out / val_out for the sparsify calls, in pairs.
+ * 0 (the default) means "d".  Process-wide; returns GK_ERR_CAPACITY if cap < 0. */
+int gk_set_capacity(int64_t cap);
+
+/* Create (or grow) the workspace of (current device, stream) for vectors of up
+ * to d elements in up to S segments.  Synchronous; call outside timed regions
+ * and before stream capture. */
+int gk_reserve(int64_t d, int32_t S, gk_stream_t stream);
+
+/* Bytes of scratch workspace a call with these sizes uses. */
+int64_t gk_workspace_bytes(int64_t d, int32_t S);
+
+/* Synchronise `stream` and copy the record of the last gk_sparsify (or the S
+ * records of the last gk_sparsify_segmented) enqueued on it to HOST memory. */
+int gk_last_stats(gk_stream_t stream, gk_stats* host_out);
+int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out);
+
+/* Number of kernels the library has launched so far in this process. */
+int64_t gk_launch_count(void);
+
+/* Text for a gk_status; the CUDA error string of the last GK_ERR_CUDA. */
+const char* gk_strerror(int code);
+const char* gk_last_cuda_error(void);
+
+/* Library version, major * 1000 + minor. */
+int gk_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GK_H_ */

@@ -1,0 +1,199 @@
+"""Python binding of the C ABI in include/gk.h.
+
+Argument marshalling only: every function takes torch CUDA tensors (device
+memory) or numpy arrays (the host call), hands raw pointers and the current
+CUDA stream to libgk_b200.so, and returns.  There is no CPU fallback: if the
+library is missing or no CUDA device is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libgk_b200.so")
+
+GK_DEV_TRUNCATED = 1
+GK_DEV_TIMEOUT = 2
+GK_DEV_BAD_SEGMENTS = 4
+
+EXPORTS = [
+    "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
+    "gk_set_capacity", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
+    "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
+]
+
+
+class GkStats(C.Structure):
+    _fields_ = [
+        ("mu", C.c_double), ("sigma", C.c_double), ("z", C.c_double), ("thres0", C.c_double),
+        ("thr_final", C.c_double), ("counts", C.c_int64 * 4), ("rounds", C.c_int32),
+        ("status", C.c_int32), ("nnz", C.c_int64), ("emitted", C.c_int64),
+    ]
+
+
+@dataclass
+class Stats:
+    mu: float
+    sigma: float
+    z: float
+    thres0: float
+    thr_final: float
+    counts: List[int]
+    rounds: int
+    status: int
+    nnz: int
+    emitted: int
+
+    @staticmethod
+    def of(s: GkStats) -> "Stats":
+        return Stats(s.mu, s.sigma, s.z, s.thres0, s.thr_final, [int(c) for c in s.counts][: max(int(s.rounds), 0)],
+                     int(s.rounds), int(s.status), int(s.nnz), int(s.emitted))
+
+
+class GkError(RuntimeError):
+    pass
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load() -> C.CDLL:
+    """Load libgk_b200.so (built by paper_1911_08772_b200/build.py).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise GkError(f"{LIB_PATH} not found: run `python -m paper_1911_08772_b200.build` first "
+                      "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int32
+    L.gk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.gk_sparsify_segmented.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.topk_exact.argtypes = [vp, i64, i64, vp, vp, vp]
+    L.topk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.gk_sparsify_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, C.POINTER(GkStats)]
+    L.gk_set_capacity.argtypes = [i64]
+    L.gk_reserve.argtypes = [i64, i32, vp]
+    L.gk_workspace_bytes.argtypes = [i64, i32]
+    L.gk_workspace_bytes.restype = i64
+    L.gk_last_stats.argtypes = [vp, C.POINTER(GkStats)]
+    L.gk_last_segment_stats.argtypes = [vp, i32, C.POINTER(GkStats)]
+    L.gk_launch_count.argtypes = []
+    L.gk_launch_count.restype = i64
+    L.gk_strerror.argtypes = [C.c_int]
+    L.gk_strerror.restype = C.c_char_p
+    L.gk_last_cuda_error.argtypes = []
+    L.gk_last_cuda_error.restype = C.c_char_p
+    L.gk_version.argtypes = []
+    for name in ("gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
+                 "gk_set_capacity", "gk_reserve", "gk_last_stats", "gk_last_segment_stats", "gk_version"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        L = load()
+        msg = L.gk_strerror(rc).decode()
+        if rc == -6:
+            msg += ": " + L.gk_last_cuda_error().decode()
+        raise GkError(f"gk error {rc}: {msg}")
+
+
+def _stream() -> int:
+    import torch
+    return int(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t, dtype) -> int:
+    import torch
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise GkError("expected a CUDA tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise GkError(f"expected a contiguous {dtype} tensor, got {t.dtype}")
+    return t.data_ptr()
+
+
+def gk_sparsify(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
+    """Enqueue one Gaussian_k error-compensated step on the current stream (see gk.h)."""
+    import torch
+    d = g.numel()
+    _check(load().gk_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), d, k,
+                              _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
+                              _dev(nnz_out, torch.int64), _stream()))
+
+
+def gk_sparsify_segmented(g, eps, seg_offsets, seg_k, idx_out, val_out, seg_nnz_out, nnz_out) -> None:
+    import torch
+    d = g.numel()
+    S = seg_offsets.numel() - 1
+    _check(load().gk_sparsify_segmented(
+        _dev(g, torch.float32), _dev(eps, torch.float32), d, _dev(seg_offsets, torch.int64),
+        _dev(seg_k, torch.int64), S, _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
+        None if seg_nnz_out is None else _dev(seg_nnz_out, torch.int64), _dev(nnz_out, torch.int64), _stream()))
+
+
+def topk_exact(u, k: int, idx_out, val_out) -> None:
+    import torch
+    _check(load().topk_exact(_dev(u, torch.float32), u.numel(), k, _dev(idx_out, torch.int32),
+                             _dev(val_out, torch.float32), _stream()))
+
+
+def topk_sparsify(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
+    import torch
+    _check(load().topk_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), g.numel(), k,
+                                _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
+                                _dev(nnz_out, torch.int64), _stream()))
+
+
+def gk_sparsify_host(g, eps, k: int, idx_out, val_out):
+    """Host-buffer step.  g, eps, idx_out, val_out: numpy arrays or CPU torch tensors
+    (pinned for speed).  eps is updated in place.  Returns (nnz, Stats)."""
+    def ptr(a):
+        return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+    d = g.numel() if hasattr(g, "numel") else g.size
+    nnz = C.c_int64(0)
+    st = GkStats()
+    _check(load().gk_sparsify_host(ptr(g), ptr(eps), d, k, ptr(idx_out), ptr(val_out),
+                                   C.addressof(nnz), C.byref(st)))
+    return int(nnz.value), Stats.of(st)
+
+
+def gk_set_capacity(cap: int) -> None:
+    _check(load().gk_set_capacity(cap))
+
+
+def gk_reserve(d: int, S: int = 1) -> None:
+    _check(load().gk_reserve(d, S, _stream()))
+
+
+def gk_workspace_bytes(d: int, S: int = 1) -> int:
+    return int(load().gk_workspace_bytes(d, S))
+
+
+def gk_last_stats() -> Stats:
+    st = GkStats()
+    _check(load().gk_last_stats(_stream(), C.byref(st)))
+    return Stats.of(st)
+
+
+def gk_last_segment_stats(S: int) -> List[Stats]:
+    arr = (GkStats * S)()
+    _check(load().gk_last_segment_stats(_stream(), S, arr))
+    return [Stats.of(s) for s in arr]
+
+
+def gk_launch_count() -> int:
+    return int(load().gk_launch_count())
+
+
+def gk_version() -> int:
+    return int(load().gk_version())
+
+
+def gk_strerror(code: int) -> str:
+    return load().gk_strerror(code).decode()

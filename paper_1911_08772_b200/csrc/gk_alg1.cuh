@@ -1,0 +1,111 @@
+// Scalar part of Algorithm 1 (arXiv 1911.08772) as device functions: the normal
+// quantile, statistics -> candidate thresholds, and the replay of the
+// count-and-adjust loop on counts taken for all candidates at once.
+#pragma once
+
+#include <math.h>
+
+#include "gk_common.cuh"
+
+namespace gk {
+
+// z with P(Z > z) = q for a standard normal Z, 0 < q < 1: Newton's iteration on
+// erfc(z / sqrt 2) / 2 - q (derivative -phi(z)), started from the leading term
+// of the tail expansion.
+__host__ __device__ inline double normal_quantile_upper(double q) {
+    if (!(q > 0.0)) return INFINITY;
+    if (!(q < 1.0)) return -INFINITY;
+    if (q == 0.5) return 0.0;
+    const bool flip = q > 0.5;
+    if (flip) q = 1.0 - q;
+    double z = sqrt(-2.0 * log(q));
+    if (z > 1.0) z -= log(z * 2.5066282746310002) / z;  // q ~ phi(z) / z
+    const double inv_sqrt2 = 0.70710678118654752440, inv_sqrt2pi = 0.39894228040143267794;
+    for (int it = 0; it < 100; ++it) {
+        const double f = 0.5 * erfc(z * inv_sqrt2) - q;
+        const double phi = inv_sqrt2pi * exp(-0.5 * z * z);
+        const double zn = z + f / phi;
+        const bool done = fabs(zn - z) <= 2e-16 * fabs(zn);
+        z = zn;
+        if (done) break;
+    }
+    return flip ? -z : z;
+}
+
+// Where one run of Algorithm 1 keeps its scalars.
+struct Alg1State {
+    gk_stats* stats;
+    double* cand64;              // kNumCand
+    float* cand32;               // kNumCand
+    unsigned long long* counts;  // kNumCand
+    float* thr_sel;
+};
+
+#ifdef __CUDACC__
+// s1 = sum(u - c), s2 = sum((u - c)^2) over the n elements, c the pivot.
+// One thread.  k >= n means p = 1 - k/n <= 0: the quantile is -inf and every
+// element passes; no statistics are needed.
+__device__ inline void alg1_thresholds(const Alg1State& a, double s1, double s2, double c, int64_t n,
+                                       int64_t k, double z) {
+    gk_stats st;
+    st.status = GK_DEV_OK;
+    st.emitted = 0;
+    for (int i = 0; i < kMaxRounds; ++i) st.counts[i] = 0;
+    for (int i = 0; i < kNumCand; ++i) a.counts[i] = 0ull;
+    if (k >= n) {
+        st.mu = st.sigma = __longlong_as_double(0x7ff8000000000000ll);
+        st.z = st.thres0 = st.thr_final = -INFINITY;
+        st.rounds = 0;
+        st.nnz = n;
+        *a.thr_sel = -INFINITY;
+        *a.stats = st;
+        return;
+    }
+    const double dn = (double)n;
+    const double mean_shift = s1 / dn;
+    double var = (s2 - s1 * mean_shift) / (dn - 1.0);  // sample variance
+    if (var < 0.0) var = 0.0;
+    st.mu = c + mean_shift;
+    st.sigma = sqrt(var);
+    st.z = z;
+    st.thres0 = st.mu + st.sigma * z;
+    st.thr_final = st.thres0;
+    st.rounds = 0;
+    st.nnz = 0;
+    *a.stats = st;
+    double tb = st.thres0;
+    for (int b = 0; b < kMaxRounds; ++b) {
+        double t = tb;
+        for (int h = 0; h + b < kMaxRounds; ++h) {
+            a.cand64[cand_index(h, b)] = t;
+            // for fp32 x and fp64 t:  x > t  <=>  x > (t rounded toward -inf to fp32)
+            a.cand32[cand_index(h, b)] = __double2float_rd(t);
+            t *= 0.5;
+        }
+        tb *= 1.5;
+    }
+    *a.thr_sel = __double2float_rd(st.thres0);
+}
+
+// Replay of the loop of Algorithm 1 on the candidate counts.  One thread.
+__device__ inline void alg1_resolve(const Alg1State& a, int64_t k) {
+    gk_stats st = *a.stats;
+    if (st.rounds == 0 && st.thr_final == -INFINITY) return;  // everything selected
+    int h = 0, b = 0;
+    for (int r = 0; r < kMaxRounds; ++r) {
+        const int ci = cand_index(h, b);
+        const long long est = (long long)__ldcg(&a.counts[ci]);
+        st.counts[r] = est;
+        st.rounds = r + 1;
+        st.thr_final = a.cand64[ci];  // the mask of this round is the last one evaluated
+        st.nnz = est;
+        *a.thr_sel = a.cand32[ci];
+        if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
+        else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
+        else break;
+    }
+    *a.stats = st;
+}
+#endif
+
+}  // namespace gk

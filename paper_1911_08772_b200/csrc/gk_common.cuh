@@ -1,0 +1,134 @@
+// Shared declarations of the CUDA library: workspace layout, small device
+// helpers, launch bookkeeping.  Internal; the public interface is include/gk.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gk.h"
+
+namespace gk {
+
+// ---------------------------------------------------------------------------
+// Algorithm 1 visits at most four thresholds, each thres0 * 0.5^a * 1.5^b with
+// a + b <= 3.  Halving is exact in binary floating point, so the ten products
+// do not depend on the order of the adjustments and can all be counted in one
+// pass.  Candidate (a, b) lives at index cand_index(a, b).
+// ---------------------------------------------------------------------------
+constexpr int kMaxRounds = 4;
+constexpr int kNumCand = 10;
+__host__ __device__ constexpr int cand_index(int a, int b) {
+    // b = 0: 0..3, b = 1: 4..6, b = 2: 7..8, b = 3: 9
+    return (b == 0 ? 0 : b == 1 ? 4 : b == 2 ? 7 : 9) + a;
+}
+
+// Compaction tile: kCompactThreads threads, kCompactRows float4 per thread.
+constexpr int kCompactThreads = 256;
+constexpr int kCompactRows = 8;
+constexpr int kCompactTileElems = kCompactThreads * kCompactRows * 4;  // 8192
+
+constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
+
+// Bounded waits: polls of a predecessor's status word before giving up.
+constexpr int kLookbackPollLimit = 1 << 22;
+
+// Tile status word of the decoupled look-back: flag in bits 63..62, payload below.
+constexpr unsigned long long kFlagShift = 62;
+constexpr unsigned long long kFlagAggregate = 1ull;
+constexpr unsigned long long kFlagPrefix = 2ull;
+constexpr unsigned long long kPayloadMask = (1ull << kFlagShift) - 1ull;
+
+// Control block at the start of every workspace.  Zeroed when the workspace is
+// created; the tickets are reset by the CTA that retires last, so every call
+// finds them at zero.
+struct Ctrl {
+    unsigned int ticket_a;     // CTAs of the accumulate kernel that have finished
+    unsigned int ticket_b;     // CTAs of the count kernel that have finished
+    unsigned int tile_ticket;  // next compaction tile to hand out
+    unsigned int ticket_h;     // CTAs of a histogram kernel that have finished
+    unsigned long long counts[kNumCand];  // #{|u| > cand}, filled by the count kernel
+    double cand64[kNumCand];              // candidate thresholds, fp64
+    float cand32[kNumCand];               // the same rounded toward -inf to fp32
+    float thr_sel;                        // threshold of the mask to return (fp32, rounded down)
+    gk_stats stats;
+    // exact Top_k state
+    unsigned int key_prefix;       // magnitude bits fixed so far
+    unsigned int key_threshold;    // final k-th largest magnitude key
+    unsigned long long need;       // how many still to take among keys matching the prefix
+    unsigned long long need_eq;    // how many entries equal to the threshold key to take
+};
+
+struct Workspace {
+    void* base = nullptr;          // device allocation
+    size_t bytes = 0;
+    int64_t d_cap = 0;             // sizes the allocation was made for
+    int32_t s_cap = 0;
+    Ctrl* ctrl = nullptr;
+    double2* partials = nullptr;            // kMaxPartials
+    unsigned long long* tile_status = nullptr;  // one per compaction tile
+    unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
+    // segmented call
+    void* seg_block = nullptr;
+    int sm_count = 0;
+};
+
+// host side (gk_host.cu)
+int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out);
+int cuda_fail(cudaError_t e);   // records the error text, returns GK_ERR_CUDA
+void note_launch(int n = 1);
+int64_t output_capacity(int64_t d);
+
+inline int64_t num_compact_tiles(int64_t d) {
+    return (d + kCompactTileElems - 1) / kCompactTileElems;
+}
+
+#define GK_CUDA_TRY(expr)                                  \
+    do {                                                   \
+        cudaError_t e__ = (expr);                          \
+        if (e__ != cudaSuccess) return ::gk::cuda_fail(e__); \
+    } while (0)
+
+// ---------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Streaming 128-bit load: the line is not expected to be read again.
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+
+__device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_status(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Deterministic block reduction of (s, q) pairs: warp shuffles, then a fixed
+// order over the warps.  Result valid in thread 0.
+template <int THREADS>
+__device__ __forceinline__ double2 block_sum2(double s, double q, double2* smem /* THREADS/32 */) {
+    s = warp_sum(s);
+    q = warp_sum(q);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) smem[w] = make_double2(s, q);
+    __syncthreads();
+    double2 r = make_double2(0.0, 0.0);
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < THREADS / 32; ++i) { r.x += smem[i].x; r.y += smem[i].y; }
+    }
+    __syncthreads();
+    return r;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace gk

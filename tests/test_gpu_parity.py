@@ -1,0 +1,315 @@
+"""GPU-vs-oracle parity through the C ABI: small sizes element by element (several
+tiles and ragged tails), edge cases, and the five workload families at full size."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_1911_08772_b200 import binding as gk
+from paper_1911_08772_b200 import workloads as wl
+
+from gpu_util import DeviceStep, bits, check_gk_step, check_segmented_step, check_topk
+
+pytestmark = pytest.mark.gpu
+
+TILE = 8192  # compaction tile of the library, to place sizes around its edges
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    from paper_1911_08772_b200 import build
+    build.build()
+    gk.load()
+    gk.gk_set_capacity(0)
+    yield
+
+
+# ------------------------------------------------------------------ small sizes, every boundary
+SMALL_D = [1, 2, 3, 4, 5, 7, 8, 31, 32, 33, 127, 128, 129, 1023, 1024, 1025, 4095, 4096, 4097,
+           TILE - 1, TILE, TILE + 1, 2 * TILE + 3, 5 * TILE - 2, 100_003]
+
+
+@pytest.mark.parametrize("d", SMALL_D)
+def test_gk_sparsify_small_sizes(d):
+    rng = wl.misc_rng(1000 + d)
+    g = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    e = (rng.standard_normal(d) * 2e-3).astype(np.float32)
+    step = DeviceStep(d)
+    for k in sorted({1, max(1, d // 100), max(1, d // 7), d}):
+        check_gk_step(step, g, e, k)
+
+
+def test_gk_sparsify_special_values():
+    d = 3 * TILE + 1
+    rng = wl.misc_rng(7)
+    g = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    e = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    g[:6] = np.array([0.0, -0.0, -0.0, 1e-45, 1e-39, 2.5], dtype=np.float32)
+    e[:6] = np.array([-0.0, -0.0, 0.0, 1e-45, -1e-39, -2.5], dtype=np.float32)
+    step = DeviceStep(d)
+    eps_new, st = check_gk_step(step, g, e, 25)
+    assert bits(eps_new)[1] == 0x80000000   # -0 + -0 = -0 survives, denormals are not flushed
+    assert bits(eps_new)[3] == 2
+    # all zeros: sigma = 0, threshold 0, nothing selected
+    z = np.zeros(d, dtype=np.float32)
+    _, st = check_gk_step(step, z, z, 10)
+    assert st.nnz == 0 and st.sigma == 0.0
+    # constant vector: sigma = 0
+    c = np.full(d, 0.375, dtype=np.float32)
+    check_gk_step(step, c, z, 10, check_counts=False)
+    # large mean relative to the spread
+    check_gk_step(step, (g + np.float32(0.5)).astype(np.float32), z, 30)
+    # negative threshold: mean far below zero selects everything
+    _, st = check_gk_step(step, (g - np.float32(5.0)).astype(np.float32), z, 30)
+    assert st.nnz == d
+
+
+def test_gk_hand_built_branch_cases():
+    # the same level vectors that pin the oracle's branch sequences
+    from test_oracle_pins import _branch_cases, _levels_vector
+    for name, d, k, levels, rounds, counts, fn, fd, nnz in _branch_cases():
+        u = _levels_vector(d, levels, seed=11)
+        step = DeviceStep(d)
+        _, st = check_gk_step(step, u, np.zeros(d, np.float32), k)
+        assert st.rounds == rounds and st.counts == counts and st.nnz == nnz, name
+        assert abs(st.thr_final / st.thres0 - fn / fd) < 1e-15
+
+
+def test_gk_capacity_truncation():
+    d = 4 * TILE + 5
+    u = wl.normal(d, 1.0, step=2)
+    z = np.zeros(d, dtype=np.float32)
+    try:
+        gk.gk_set_capacity(37)
+        step = DeviceStep(d, cap=37)
+        eps_new, st = check_gk_step(step, u, z, 500)
+        assert st.status & gk.GK_DEV_TRUNCATED and st.emitted == 37 and st.nnz > 37
+    finally:
+        gk.gk_set_capacity(0)
+
+
+def test_gk_is_deterministic_and_stateless():
+    d = 1_000_003
+    g = wl.laplace_mixture(d, step=3)
+    e = wl.normal(d, 1e-4, step=4)
+    step = DeviceStep(d)
+    outs = []
+    for _ in range(3):
+        eps_new, st = check_gk_step(step, g, e, 1001)
+        outs.append((bits(eps_new).copy(), st.thr_final, st.mu, st.sigma, st.nnz))
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0]) and o[1:] == outs[0][1:]
+
+
+def test_gk_on_a_side_stream():
+    d = 300_007
+    g = wl.normal(d, 1e-3, step=11)
+    z = np.zeros(d, np.float32)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        step = DeviceStep(d)
+        check_gk_step(step, g, z, 301)
+
+
+# ------------------------------------------------------------------ exact Top_k
+@pytest.mark.parametrize("d", [1, 2, 5, 33, 1025, TILE, TILE + 1, 3 * TILE + 2, 250_001])
+def test_topk_small_sizes(d):
+    rng = wl.misc_rng(2000 + d)
+    u = rng.standard_normal(d).astype(np.float32)
+    for k in sorted({1, max(1, d // 50), max(1, d // 3), d}):
+        check_topk(u, k)
+
+
+def test_topk_ties_and_zeros():
+    rng = wl.misc_rng(5)
+    d = 2 * TILE + 77
+    u = (np.round(rng.standard_normal(d) * 2) / 2).astype(np.float32)  # heavy ties, many +-0
+    u[::3] *= -1
+    for k in (1, 10, 500, d // 2, d - 1, d):
+        check_topk(u, k)
+    z = np.zeros(d, dtype=np.float32)
+    z[1::2] = -0.0
+    idx, _ = check_topk(z, 100)
+    assert idx.tolist() == list(range(100))
+    same = np.full(d, -3.5, dtype=np.float32)
+    idx, _ = check_topk(same, 1000)
+    assert idx.tolist() == list(range(1000))
+    tiny = np.array([1e-45, -1e-45, 0.0, 3e-39, -3e38], dtype=np.float32)
+    check_topk(tiny, 3)
+
+
+def test_topk_sparsify_matches_eq2_with_exact_topk():
+    d = 3 * TILE + 9
+    g = wl.laplace(d, 1.0, step=21)
+    e = wl.normal(d, 0.5, step=22)
+    k = 123
+    dev = torch.device("cuda:0")
+    dg, de = torch.from_numpy(g).to(dev), torch.from_numpy(e).to(dev)
+    idx = torch.empty(k, dtype=torch.int32, device=dev)
+    val = torch.empty(k, dtype=torch.float32, device=dev)
+    nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+    gk.topk_sparsify(dg, de, k, idx, val, nnz)
+    torch.cuda.synchronize()
+    u = orc.accumulate(g, e)
+    oi, ov = orc.topk_exact(u, k)
+    assert int(nnz.item()) == k
+    assert np.array_equal(idx.cpu().numpy(), oi) and np.array_equal(bits(val.cpu().numpy()), bits(ov))
+    assert np.array_equal(bits(de.cpu().numpy()), bits(orc.residual(u, oi, ov)))
+
+
+# ------------------------------------------------------------------ segmented
+def _dev_i64(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int64)).to("cuda:0")
+
+
+def test_segmented_small_and_ragged():
+    offsets = np.array([0, 1, 1, 3, 10, 64, 65, 1000, 1003, 5000, 5000, 9001, 3 * TILE + 6, 4 * TILE + 1],
+                       dtype=np.int64)
+    d = int(offsets[-1])
+    S = offsets.shape[0] - 1
+    rng = wl.misc_rng(31)
+    g = (rng.standard_normal(d) * np.repeat(rng.uniform(1e-4, 1e-1, S), np.diff(offsets))).astype(np.float32)
+    e = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    sizes = np.diff(offsets)
+    step = DeviceStep(d)
+    nn = torch.zeros(S, dtype=torch.int64, device="cuda:0")
+    for rho_num, rho_den in ((1, 100), (1, 3), (1, 1)):
+        seg_k = np.array([max(1, wl.ceil_k(int(n), rho_num, rho_den)) for n in sizes], dtype=np.int64)
+        check_segmented_step(step, g, e, offsets, seg_k, _dev_i64(offsets), _dev_i64(seg_k), nn)
+
+
+def test_segmented_single_segment_equals_whole_vector():
+    d = 2 * TILE + 11
+    g = wl.normal(d, 1e-2, step=5)
+    z = np.zeros(d, np.float32)
+    offsets = np.array([0, d], dtype=np.int64)
+    seg_k = np.array([50], dtype=np.int64)
+    step = DeviceStep(d)
+    nn = torch.zeros(1, dtype=torch.int64, device="cuda:0")
+    eps_a, sts = check_segmented_step(step, g, z, offsets, seg_k, _dev_i64(offsets), _dev_i64(seg_k), nn)
+    eps_b, st = check_gk_step(step, g, z, 50)
+    assert np.array_equal(bits(eps_a), bits(eps_b))
+    assert sts[0].thr_final == st.thr_final or abs(sts[0].thr_final / st.thr_final - 1) < 1e-12
+
+
+def test_segmented_bad_table_is_reported_not_fatal():
+    d = 20_000
+    g = wl.normal(d, 1e-2, step=6)
+    offsets = np.array([0, 9000, 8000, d], dtype=np.int64)  # not ascending
+    seg_k = np.array([5, 5, 5], dtype=np.int64)
+    step = DeviceStep(d)
+    step.g.copy_(torch.from_numpy(g))
+    step.eps.zero_()
+    step.arm()
+    nn = torch.zeros(3, dtype=torch.int64, device="cuda:0")
+    gk.gk_sparsify_segmented(step.g, step.eps, _dev_i64(offsets), _dev_i64(seg_k), step.idx[:d], step.val[:d],
+                             nn, step.nnz[:1])
+    idx, val, n = step.outputs()
+    sts = gk.gk_last_segment_stats(3)
+    assert n == 0 and all(s.status & gk.GK_DEV_BAD_SEGMENTS for s in sts)
+
+
+# ------------------------------------------------------------------ the workload families, full size
+def _ec_loop(w, rho, steps, check_every=1, also=None):
+    k = w.k(rho)
+    step = DeviceStep(w.d)
+    eps = np.zeros(w.d, dtype=np.float32)
+    g = np.empty(w.d, dtype=np.float32)
+    for t in range(steps):
+        w.grad(t, g)
+        eps, st = check_gk_step(step, g, eps, k)
+        if also is not None:
+            also(t, st)
+    return eps
+
+
+def test_workload_resnet20_normal():
+    w = wl.resnet20_normal()
+    assert w.k("1e-3") == 270
+    _ec_loop(w, "1e-3", 1 + 10)
+
+
+def test_workload_vgg16_laplace_mixture_100_steps():
+    w = wl.vgg16_laplace_mixture()
+    nnzs = []
+    _ec_loop(w, "1e-3", 100, also=lambda t, st: nnzs.append(st.nnz))
+    assert min(nnzs) > 0
+
+
+@pytest.mark.parametrize("rho", ["1e-3", "1e-2"])
+def test_workload_resnet50_global_and_segmented(rho):
+    w = wl.resnet50_segmented()
+    part = w.partition
+    assert part.S == 161 and int(part.sizes().min()) >= 64
+    steps = 20
+    # global selection
+    _ec_loop(w, rho, steps)
+    # layer-wise selection
+    seg_k = part.seg_k(*wl.RHO[rho])
+    step = DeviceStep(w.d)
+    dev_off, dev_k = _dev_i64(part.offsets), _dev_i64(seg_k)
+    nn = torch.zeros(part.S, dtype=torch.int64, device="cuda:0")
+    eps = np.zeros(w.d, dtype=np.float32)
+    g = np.empty(w.d, dtype=np.float32)
+    for t in range(steps):
+        w.grad(t, g)
+        eps, _ = check_segmented_step(step, g, eps, part.offsets, seg_k, dev_off, dev_k, nn)
+
+
+@pytest.mark.parametrize("rho", ["1e-3", "5e-3"])
+def test_workload_lstm_student_t(rho):
+    w = wl.lstm_student_t()
+    eps = _ec_loop(w, rho, 20)
+    # exact radix Top_k on the same u (= last eps plus a fresh gradient)
+    g = w.grad(20, None)
+    u = orc.accumulate(g, eps)
+    check_topk(u, w.k(rho))
+
+
+@pytest.mark.parametrize("dist", ["normal", "laplace"])
+@pytest.mark.parametrize("log2d", [20, 22, 24, 26])
+def test_workload_sweep(dist, log2d):
+    w = wl.sweep_point(1 << log2d, dist)
+    g = w.grad(0, None)
+    z = np.zeros(w.d, dtype=np.float32)
+    step = DeviceStep(w.d)
+    for rho in w.rhos:
+        check_gk_step(step, g, z, w.k(rho))
+    for rho in w.rhos:
+        check_topk(g, w.k(rho))
+
+
+@pytest.mark.parametrize("dist", ["normal", "laplace"])
+def test_workload_sweep_largest(dist):
+    """d = 2^28 (1 GiB per vector): Gaussian_k against the oracle in full; exact Top_k by
+    properties that fix the answer uniquely (count, threshold, tie order), since a full
+    CPU sort of 2^28 keys takes most of a minute per case."""
+    w = wl.sweep_point(1 << 28, dist)
+    g = w.grad(0, None)
+    z = np.zeros(w.d, dtype=np.float32)
+    step = DeviceStep(w.d)
+    for rho in w.rhos:
+        check_gk_step(step, g, z, w.k(rho))
+    del step
+    torch.cuda.empty_cache()
+    k = w.k("1e-3")
+    dev = torch.device("cuda:0")
+    du = torch.from_numpy(g).to(dev)
+    idx = torch.empty(k, dtype=torch.int32, device=dev)
+    val = torch.empty(k, dtype=torch.float32, device=dev)
+    gk.topk_exact(du, k, idx, val)
+    torch.cuda.synchronize()
+    hi, hv = idx.cpu().numpy(), val.cpu().numpy()
+    assert np.all(np.diff(hi) > 0)
+    assert np.array_equal(bits(hv), bits(g[hi]))
+    kth = np.abs(hv).min()
+    # everything strictly above the k-th magnitude is in; nothing below it is
+    assert orc.count_above(g, float(kth)) == int((np.abs(hv) > kth).sum())
+    below = np.nextafter(kth, np.float32(0))
+    assert orc.count_above(g, float(below)) >= k
+    # entries equal to the k-th magnitude are the lowest-index ones
+    ties_all = np.nonzero(np.abs(g) == kth)[0]
+    ties_sel = hi[np.abs(hv) == kth]
+    assert np.array_equal(ties_sel, ties_all[:ties_sel.size].astype(np.int32))
