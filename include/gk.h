@@ -166,6 +166,18 @@ int64_t gk_workspace_bytes(int64_t d, int32_t S);
 int gk_last_stats(gk_stream_t stream, gk_stats* host_out);
 int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out);
 
+/*
+ * Per-stage device timing (tracing aid, off by default; process-wide switch).
+ * While enabled, every call records a CUDA event on its stream before its first
+ * kernel and after each kernel.  gk_last_stage_ms synchronises the stream and
+ * writes the durations in milliseconds of the stages of the last call enqueued on
+ * it to HOST ms_out[0..*n_stages-1] (at most 5: gk_sparsify has accumulate, count,
+ * compact; topk_exact has three histogram passes and compact; topk_sparsify has
+ * accumulate first).
+ */
+int gk_stage_timing(int enable);
+int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages);
+
 /* Number of kernels the library has launched so far in this process. */
 int64_t gk_launch_count(void);
 

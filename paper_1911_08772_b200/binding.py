@@ -22,7 +22,7 @@ GK_DEV_BAD_SEGMENTS = 4
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
     "gk_set_capacity", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
-    "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
+    "gk_stage_timing", "gk_last_stage_ms", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
 ]
 
 
@@ -81,6 +81,10 @@ def load() -> C.CDLL:
     L.gk_workspace_bytes.restype = i64
     L.gk_last_stats.argtypes = [vp, C.POINTER(GkStats)]
     L.gk_last_segment_stats.argtypes = [vp, i32, C.POINTER(GkStats)]
+    L.gk_stage_timing.argtypes = [C.c_int]
+    L.gk_stage_timing.restype = C.c_int
+    L.gk_last_stage_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+    L.gk_last_stage_ms.restype = C.c_int
     L.gk_launch_count.argtypes = []
     L.gk_launch_count.restype = i64
     L.gk_strerror.argtypes = [C.c_int]
@@ -185,6 +189,19 @@ def gk_last_segment_stats(S: int) -> List[Stats]:
     arr = (GkStats * S)()
     _check(load().gk_last_segment_stats(_stream(), S, arr))
     return [Stats.of(s) for s in arr]
+
+
+def gk_stage_timing(enable: bool) -> None:
+    _check(load().gk_stage_timing(int(enable)))
+
+
+def gk_last_stage_ms() -> List[float]:
+    """Durations (ms) of the stages of the last call on the current stream; needs
+    gk_stage_timing(True) before that call.  Synchronises the stream."""
+    ms = (C.c_float * 5)()
+    n = C.c_int(0)
+    _check(load().gk_last_stage_ms(_stream(), ms, C.byref(n)))
+    return [float(ms[i]) for i in range(n.value)]
 
 
 def gk_launch_count() -> int:

@@ -70,12 +70,17 @@ struct Workspace {
     // segmented call
     void* seg_block = nullptr;
     int sm_count = 0;
+    // per-stage timing (tracing aid)
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    int n_stages = 0;
 };
 
 // host side (gk_host.cu)
 int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out);
 int cuda_fail(cudaError_t e);   // records the error text, returns GK_ERR_CUDA
 void note_launch(int n = 1);
+// Stage timing: mark(ws, st, i) records event i (0 = before the first kernel) when tracing is on.
+void stage_mark(Workspace* ws, cudaStream_t st, int i);
 int64_t output_capacity(int64_t d);
 
 inline int64_t num_compact_tiles(int64_t d) {

@@ -29,6 +29,15 @@ int cuda_fail(cudaError_t e) {
 
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+static std::atomic<int> g_stage_timing{0};
+
+void stage_mark(Workspace* ws, cudaStream_t st, int i) {
+    if (!g_stage_timing.load(std::memory_order_relaxed) || i < 0 || i > 5) return;
+    if (!ws->ev[i] && cudaEventCreate(&ws->ev[i]) != cudaSuccess) { cudaGetLastError(); return; }
+    cudaEventRecord(ws->ev[i], st);
+    ws->n_stages = i;
+}
+
 int64_t output_capacity(int64_t d) {
     const int64_t c = g_capacity.load(std::memory_order_relaxed);
     return c > 0 ? c : d;
@@ -153,6 +162,22 @@ extern "C" int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* ho
         host_out[s].status |= total.status;
         if (!(total.status & (GK_DEV_TRUNCATED | GK_DEV_TIMEOUT))) host_out[s].emitted = host_out[s].nnz;
     }
+    return GK_OK;
+}
+
+extern "C" int gk_stage_timing(int enable) {
+    g_stage_timing.store(enable ? 1 : 0);
+    return GK_OK;
+}
+
+extern "C" int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages) {
+    if (!ms_out || !n_stages) return GK_ERR_NULL;
+    Workspace* ws = find_workspace((cudaStream_t)stream);
+    if (!ws) return GK_ERR_NULL;
+    GK_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    *n_stages = ws->n_stages;
+    for (int i = 0; i < ws->n_stages; ++i)
+        GK_CUDA_TRY(cudaEventElapsedTime(&ms_out[i], ws->ev[i], ws->ev[i + 1]));
     return GK_OK;
 }
 

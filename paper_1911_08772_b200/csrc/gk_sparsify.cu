@@ -209,18 +209,22 @@ int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, in
         z = normal_quantile_upper(1.0 - p);
     }
     const int grid_a = reduction_grid(ws, d, kAccThreads, kAccUnroll, 4);
+    stage_mark(ws, st, 0);
     k_accumulate_stats<<<grid_a, kAccThreads, 0, st>>>(g, eps, d, k, z, ws->ctrl, ws->partials,
                                                        ws->tile_status, n_tiles);
     note_launch();
+    stage_mark(ws, st, 1);
     if (k < d) {
         const int grid_b = reduction_grid(ws, d, kCntThreads, kCntUnroll, 4);
         k_count_candidates<<<grid_b, kCntThreads, 0, st>>>(eps, d, k, ws->ctrl);
         note_launch();
     }
+    stage_mark(ws, st, 2);
     k_compact_threshold<false><<<n_tiles, kCompactThreads, 0, st>>>(
         eps, d, ws->ctrl, ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d), nullptr, 0,
         nullptr);
     note_launch();
+    stage_mark(ws, st, 3);
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;
 }

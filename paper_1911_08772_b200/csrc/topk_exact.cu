@@ -268,14 +268,19 @@ static int hist_grid(const Workspace* ws, int64_t d) {
 
 template <bool CLEAR>
 static int enqueue_topk(Workspace* ws, float* u, int64_t d, int64_t k, int32_t* idx_out, float* val_out,
-                        cudaStream_t st) {
+                        cudaStream_t st, int ev0) {
     const int n_tiles = (int)num_compact_tiles(d);
     const int grid = hist_grid(ws, d);
+    stage_mark(ws, st, ev0);
     k_radix_histogram<0><<<grid, kHistThreads, 0, st>>>(u, d, k, ws->ctrl, ws->hist, ws->tile_status, n_tiles);
+    stage_mark(ws, st, ev0 + 1);
     k_radix_histogram<1><<<grid, kHistThreads, 0, st>>>(u, d, k, ws->ctrl, ws->hist, ws->tile_status, n_tiles);
+    stage_mark(ws, st, ev0 + 2);
     k_radix_histogram<2><<<grid, kHistThreads, 0, st>>>(u, d, k, ws->ctrl, ws->hist, ws->tile_status, n_tiles);
+    stage_mark(ws, st, ev0 + 3);
     k_compact_topk<CLEAR><<<n_tiles, kCompactThreads, 0, st>>>(u, d, ws->ctrl, ws->tile_status, n_tiles,
                                                              idx_out, val_out);
+    stage_mark(ws, st, ev0 + 4);
     note_launch(4);
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;
@@ -294,7 +299,7 @@ extern "C" int topk_exact(const float* u, int64_t d, int64_t k, int32_t* idx_out
     Workspace* ws = nullptr;
     const int wrc = acquire_workspace(d, 1, (cudaStream_t)stream, &ws);
     if (wrc != GK_OK) return wrc;
-    return enqueue_topk<false>(ws, const_cast<float*>(u), d, k, idx_out, val_out, (cudaStream_t)stream);
+    return enqueue_topk<false>(ws, const_cast<float*>(u), d, k, idx_out, val_out, (cudaStream_t)stream, 0);
 }
 
 extern "C" int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
@@ -313,7 +318,8 @@ extern "C" int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, i
     int64_t grid = (n4 + 511) / 512;
     if (grid < 1) grid = 1;
     if (grid > (int64_t)ws->sm_count * 8) grid = (int64_t)ws->sm_count * 8;
+    stage_mark(ws, st, 0);
     k_accumulate_only<<<(int)grid, 512, 0, st>>>(g, eps, d, ws->ctrl, nnz_out, k);
     note_launch();
-    return enqueue_topk<true>(ws, eps, d, k, idx_out, val_out, st);
+    return enqueue_topk<true>(ws, eps, d, k, idx_out, val_out, st, 1);
 }

@@ -88,7 +88,7 @@ def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, c
     if k < d:
         assert rel_close(st.mu, ost.mu, 1e-6) or abs(st.mu - ost.mu) <= 1e-9 * ost.sigma
         assert rel_close(st.sigma, ost.sigma)
-        assert rel_close(st.z, ost.z, 1e-12)
+        assert abs(st.z - ost.z) <= 1e-12 * max(1.0, abs(ost.z))
         assert rel_close(st.thres0, ost.thres0) or abs(st.thres0 - ost.thres0) <= 1e-6 * ost.sigma
         assert rel_close(st.thr_final, ost.thr_final) or abs(st.thr_final - ost.thr_final) <= 1e-6 * ost.sigma, \
             (st, ost)
