@@ -183,6 +183,22 @@ def time_region(torch, fn, steps):
     return a.elapsed_time(b)
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: the job is as fast as its slowest replica."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(world: int, bytes_per_step: float, steps: int, ms: float) -> float:
+    """Aggregate over all replicas: every rank processed `steps` vectors in `ms`."""
+    return world * bytes_per_step * steps / (ms * 1e-3) / 1e9
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -237,13 +253,10 @@ def run_ours(args):
         ms = time_region(torch, step, K)
     barrier()
     launches = gk.gk_launch_count() - launches0
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(ms, world, dev)
     nnz_mean = float(nnz.item())  # of the last step; 12 * nnz is ~0.03 % of the bytes
     bytes_step = algorithmic_bytes(d, nnz_mean)
-    value = world * bytes_step * K / (ms * 1e-3) / 1e9
+    value = whole_job_gbs(world, bytes_step, K, ms)
     peak, peak_src = measured_peaks()
 
     if rank != 0:
