@@ -2,7 +2,7 @@
 """Benchmark of the error-compensated Gaussian_k sparsifier on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload NAME] [--all-configs]
+                    [--workload NAME] [--path 0|1] [--loop-only]
 
 One "step" is one whole pass of the hot path -- gk_sparsify(g, eps, d, k, ...) -- over one
 synthetic gradient vector with the residual eps carried from step to step.  The default
@@ -37,7 +37,9 @@ from paper_1911_08772_b200 import workloads as wl  # noqa: E402
 METRIC = "GaussianK sparsify GB/s (% HBM peak) at d=25.6M, rho=1e-3; speedup vs exact Top_k"
 UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
-N_ROTATE = 4  # distinct gradient buffers cycled through, so g is never L2-resident at step start
+N_ROTATE = 20   # distinct gradients: the workload's 20 error-compensation iterations, then again
+EPISODE = 20    # steps that share one residual buffer (eps starts at zero)
+MAX_EPS = 48    # residual buffers kept (pre-zeroed); beyond that they are reused as they stand
 
 
 def measured_peaks():
@@ -220,23 +222,31 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     gk.load()
+    gk.gk_set_path(args.path)
 
     w, rho = pick_workload(args.workload)
     d, k = w.d, w.k(rho)
     K, W = args.steps, max(args.warmup, 3)
 
-    # inputs resident in HBM: N_ROTATE gradient vectors (a different seed per rank)
+    # inputs resident in HBM: the gradients of N_ROTATE steps (a different seed per rank), and
+    # one zeroed residual per episode of EPISODE steps, as in the workload's EC loop
+    n_rot = N_ROTATE if 4 * d * (N_ROTATE + MAX_EPS) < 60e9 else 4
+    if args.rotate:
+        n_rot = args.rotate
     gs = []
-    for j in range(N_ROTATE):
-        gs.append(torch.from_numpy(w.grad(1000 * rank + j, None)).to(dev))
-    eps = torch.zeros(d, dtype=torch.float32, device=dev)
+    buf = np.empty(d, dtype=np.float32)
+    for j in range(n_rot):
+        gs.append(torch.from_numpy(w.grad(1000 * rank + j, buf)).to(dev))
+    n_eps = max(1, min(MAX_EPS, (W + K + EPISODE - 1) // EPISODE)) if n_rot == N_ROTATE else 2
+    epss = [torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(n_eps)]
+    eps = epss[0]
     idx = torch.empty(d, dtype=torch.int32, device=dev)
     val = torch.empty(d, dtype=torch.float32, device=dev)
     nnz = torch.zeros(1, dtype=torch.int64, device=dev)
     gk.gk_reserve(d, 1)
 
     def step(t):
-        gk.gk_sparsify(gs[t % N_ROTATE], eps, k, idx, val, nnz)
+        gk.gk_sparsify(gs[t % n_rot], epss[(t // EPISODE) % n_eps], k, idx, val, nnz)
 
     def barrier():
         torch.cuda.synchronize()
@@ -250,7 +260,7 @@ def run_ours(args):
     launches0 = gk.gk_launch_count()
     sampler = ClockSampler(local)
     with sampler:
-        ms = time_region(torch, step, K)
+        ms = time_region(torch, lambda t: step(W + t), K)
     barrier()
     launches = gk.gk_launch_count() - launches0
     ms = max_over_ranks(ms, world, dev)
@@ -263,24 +273,45 @@ def run_ours(args):
         if world > 1:
             dist.destroy_process_group()
         return
+    if args.loop_only:
+        print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+                          "warmup": W, "ms_per_step": ms / K, "path": args.path, "loop_only": True}))
+        return
 
-    # ---- per-kernel durations (CUDA events recorded by the library between its kernels)
-    gk.gk_stage_timing(True)
-    stage = np.zeros(3)
+    # ---- per-kernel durations (CUDA events recorded by the library around its kernels)
     Ks = min(K, 200)
-    for t in range(Ks):
-        step(t)
-        stage += np.array(gk.gk_last_stage_ms()[:3])
-    gk.gk_stage_timing(False)
-    stage /= Ks
-    acc_bytes = 12.0 * d
+
+    def stage_means(n_stage):
+        acc = np.zeros(n_stage)
+        gk.gk_stage_timing(True)
+        for t in range(Ks):
+            step(W + K + t)
+            acc += np.array(gk.gk_last_stage_ms()[:n_stage])
+        gk.gk_stage_timing(False)
+        return acc / Ks
+
+    fused = stage_means(7)
+    fused_ms = float(fused[0])
     roof = {
-        "bound": "hbm", "kernel": "k_accumulate_stats", "achieved": acc_bytes / (stage[0] * 1e-3) / 1e9,
+        "bound": "hbm", "kernel": "k_gk_fused", "achieved": bytes_step / (fused_ms * 1e-3) / 1e9,
         "peak": peak, "unit": "GB/s", "peak_source": peak_src,
-        "frac": acc_bytes / (stage[0] * 1e-3) / 1e9 / peak,
-        "traffic": None,
+        "frac": bytes_step / (fused_ms * 1e-3) / 1e9 / peak,
+        "traffic": None, "kernel_ms": fused_ms,
+        "phase_ms": {"accumulate_stats+barrier": fused[1], "count_loop": fused[2], "barrier2": fused[3],
+                     "replay_rounds": fused[4], "compact": fused[5], "last_cta_exit": fused[6]},
+        "bytes_per_launch": bytes_step,
+    }
+    # the three-kernel path (look-back compaction) on the same steps, stage by stage
+    gk.gk_set_path(1)
+    for t in range(3):
+        step(t)
+    ms3 = time_region(torch, lambda t: step(W + t), Ks) / Ks
+    stage = stage_means(3)
+    gk.gk_set_path(0)
+    three = {
+        "ms_per_step": ms3, "gbs": bytes_step / ms3 / 1e6,
         "stage_ms": {"accumulate_stats": stage[0], "count_candidates": stage[1], "compact": stage[2]},
-        "stage_gbs": {"accumulate_stats(12d)": acc_bytes / stage[0] / 1e6,
+        "stage_gbs": {"accumulate_stats(12d)": 12.0 * d / stage[0] / 1e6,
                       "count_candidates(4d)": 4.0 * d / stage[1] / 1e6,
                       "compact(4d+12nnz)": (4.0 * d + 12 * nnz_mean) / stage[2] / 1e6},
     }
@@ -298,16 +329,16 @@ def run_ours(args):
 
     # ---- exact Top_k on the same data: operator (given u) and sparsifier (Eq. 2 with Top_k)
     Kt = min(K, 100)
-    u = eps.clone()
+    u = epss[0].clone()
     tk_idx = torch.empty(k, dtype=torch.int32, device=dev)
     tk_val = torch.empty(k, dtype=torch.float32, device=dev)
     for _ in range(3):
         gk.topk_exact(u, k, tk_idx, tk_val)
     ms_topk = time_region(torch, lambda t: gk.topk_exact(u, k, tk_idx, tk_val), Kt) / Kt
-    eps2 = torch.zeros_like(eps)
+    eps2 = torch.zeros_like(epss[0])
     for t in range(3):
-        gk.topk_sparsify(gs[t % N_ROTATE], eps2, k, tk_idx, tk_val, nnz)
-    ms_topk_sp = time_region(torch, lambda t: gk.topk_sparsify(gs[t % N_ROTATE], eps2, k, tk_idx, tk_val, nnz),
+        gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz)
+    ms_topk_sp = time_region(torch, lambda t: gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz),
                              Kt) / Kt
     del eps2, u
 
@@ -346,13 +377,15 @@ def run_ours(args):
         "config": {
             "workload": f"{w.name} d={d} rho={rho} k={k} whole-vector selection, eps carried over",
             "l2": f"inputs per step g+eps = {8 * d / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2; "
-                  f"{N_ROTATE} gradient buffers in rotation; no flush in the headline loop",
+                  f"{n_rot} gradient and {n_eps} residual buffers in rotation "
+                  f"(episodes of {EPISODE} steps from eps = 0); no flush in the headline loop",
+            "path": "fused cooperative kernel (1 launch per step)",
             "bytes_per_step": bytes_step, "nnz_last_step": nnz_mean,
             "parallelism": "replicas only" if world > 1 else "single GPU",
         },
         "pct_of_hbm_peak": {"measured_copy": value / world / peak, "nominal_8TBs": value / world / 8000.0},
         "elements_per_s": world * d * K / (ms * 1e-3),
-        "roofline": roof,
+        "roofline": roof, "three_kernel_path": three,
         "cold_l2": {"ms_per_step": statistics.median(cold), "gbs": bytes_step / statistics.median(cold) / 1e6,
                     "note": "256 MB written between steps; per-step CUDA events"},
         "topk": {"topk_exact_ms": ms_topk, "topk_sparsify_ms": ms_topk_sp,
@@ -374,6 +407,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--path", type=int, default=0, choices=[0, 1],
+                    help="0: fused cooperative kernel, 1: three kernels with look-back")
+    ap.add_argument("--rotate", type=int, default=0,
+                    help="number of gradient buffers kept on the device (default 20; small for captures)")
+    ap.add_argument("--loop-only", action="store_true",
+                    help="run only warm-up and the timed loop (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -153,6 +153,17 @@ int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k, int32_t* 
  * 0 (the default) means "d".  Process-wide; returns GK_ERR_CAPACITY if cap < 0. */
 int gk_set_capacity(int64_t cap);
 
+/*
+ * Which implementation gk_sparsify (and gk_sparsify_host) uses.  Process-wide.
+ *   0 (default)  one persistent cooperative kernel that keeps what fits of u in
+ *                shared memory between the phases of Algorithm 1; falls back to
+ *                path 1 where cooperative launch is unavailable and for k = d.
+ *   1            three kernels: accumulate + statistics, candidate counts,
+ *                compaction by decoupled look-back.
+ * Both give identical results.  Returns GK_ERR_SIZE for any other value.
+ */
+int gk_set_path(int path);
+
 /* Create (or grow) the workspace of (current device, stream) for vectors of up
  * to d elements in up to S segments.  Synchronous; call outside timed regions
  * and before stream capture. */
@@ -171,9 +182,11 @@ int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out);
  * While enabled, every call records a CUDA event on its stream before its first
  * kernel and after each kernel.  gk_last_stage_ms synchronises the stream and
  * writes the durations in milliseconds of the stages of the last call enqueued on
- * it to HOST ms_out[0..*n_stages-1] (at most 5: gk_sparsify has accumulate, count,
- * compact; topk_exact has three histogram passes and compact; topk_sparsify has
- * accumulate first).
+ * it to HOST ms_out[0..*n_stages-1] (at most 8).  gk_sparsify, fused kernel: the
+ * kernel, then six spans from timestamps the kernel takes itself (accumulate incl.
+ * first barrier, counting loop, second barrier, replay of the rounds, compaction,
+ * exit of the last CTA); three-kernel path: accumulate, count, compact.  topk_exact:
+ * three histogram passes and compact; topk_sparsify has accumulate first.
  */
 int gk_stage_timing(int enable);
 int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages);

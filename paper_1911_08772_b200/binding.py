@@ -21,7 +21,7 @@ GK_DEV_BAD_SEGMENTS = 4
 
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
-    "gk_set_capacity", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
+    "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
 ]
 
@@ -76,6 +76,7 @@ def load() -> C.CDLL:
     L.topk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     L.gk_sparsify_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, C.POINTER(GkStats)]
     L.gk_set_capacity.argtypes = [i64]
+    L.gk_set_path.argtypes = [C.c_int]
     L.gk_reserve.argtypes = [i64, i32, vp]
     L.gk_workspace_bytes.argtypes = [i64, i32]
     L.gk_workspace_bytes.restype = i64
@@ -93,7 +94,7 @@ def load() -> C.CDLL:
     L.gk_last_cuda_error.restype = C.c_char_p
     L.gk_version.argtypes = []
     for name in ("gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
-                 "gk_set_capacity", "gk_reserve", "gk_last_stats", "gk_last_segment_stats", "gk_version"):
+                 "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_last_stats", "gk_last_segment_stats", "gk_version"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -171,6 +172,11 @@ def gk_set_capacity(cap: int) -> None:
     _check(load().gk_set_capacity(cap))
 
 
+def gk_set_path(path: int) -> None:
+    """0: fused cooperative kernel (default); 1: three kernels with look-back."""
+    _check(load().gk_set_path(path))
+
+
 def gk_reserve(d: int, S: int = 1) -> None:
     _check(load().gk_reserve(d, S, _stream()))
 
@@ -198,7 +204,7 @@ def gk_stage_timing(enable: bool) -> None:
 def gk_last_stage_ms() -> List[float]:
     """Durations (ms) of the stages of the last call on the current stream; needs
     gk_stage_timing(True) before that call.  Synchronises the stream."""
-    ms = (C.c_float * 5)()
+    ms = (C.c_float * 8)()
     n = C.c_int(0)
     _check(load().gk_last_stage_ms(_stream(), ms, C.byref(n)))
     return [float(ms[i]) for i in range(n.value)]

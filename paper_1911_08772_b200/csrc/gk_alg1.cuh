@@ -88,23 +88,27 @@ __device__ inline void alg1_thresholds(const Alg1State& a, double s1, double s2,
 }
 
 // Replay of the loop of Algorithm 1 on the candidate counts.  One thread.
-__device__ inline void alg1_resolve(const Alg1State& a, int64_t k) {
+// Returns the index of the candidate whose mask is returned (-1: everything).
+__device__ inline int alg1_resolve(const Alg1State& a, int64_t k) {
     gk_stats st = *a.stats;
-    if (st.rounds == 0 && st.thr_final == -INFINITY) return;  // everything selected
-    int h = 0, b = 0;
+    if (st.rounds == 0 && st.thr_final == -INFINITY) return -1;  // everything selected
+    int h = 0, b = 0, chosen = 0;
     for (int r = 0; r < kMaxRounds; ++r) {
         const int ci = cand_index(h, b);
-        const long long est = (long long)__ldcg(&a.counts[ci]);
+        // the counts may live in global or in shared memory: a generic volatile load serves both
+        const long long est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&a.counts[ci]);
         st.counts[r] = est;
         st.rounds = r + 1;
         st.thr_final = a.cand64[ci];  // the mask of this round is the last one evaluated
         st.nnz = est;
         *a.thr_sel = a.cand32[ci];
+        chosen = ci;
         if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
         else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
         else break;
     }
     *a.stats = st;
+    return chosen;
 }
 #endif
 

@@ -27,6 +27,7 @@ constexpr int kCompactThreads = 256;
 constexpr int kCompactRows = 8;
 constexpr int kCompactTileElems = kCompactThreads * kCompactRows * 4;  // 8192
 
+constexpr int kFusedGridCap = 512;  // upper bound on the grid of the fused kernel
 constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
 
 // Bounded waits: polls of a predecessor's status word before giving up.
@@ -56,6 +57,10 @@ struct Ctrl {
     unsigned int key_threshold;    // final k-th largest magnitude key
     unsigned long long need;       // how many still to take among keys matching the prefix
     unsigned long long need_eq;    // how many entries equal to the threshold key to take
+    // fused kernel: %globaltimer of CTA 0 at its start, after the first barrier and the
+    // thresholds, after its counting loop, after the second barrier, after the replay of the
+    // rounds, at the end of its compaction; and of the CTA that leaves last
+    unsigned long long phase_t[8];
 };
 
 struct Workspace {
@@ -67,12 +72,15 @@ struct Workspace {
     double2* partials = nullptr;            // kMaxPartials
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
+    unsigned int* cta_counts = nullptr;     // fused kernel: kFusedGridCap x kNumCand
+    unsigned int* bars = nullptr;           // fused kernel: two barrier counters and an exit counter
     // segmented call
     void* seg_block = nullptr;
     int sm_count = 0;
     // per-stage timing (tracing aid)
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     int n_stages = 0;
+    bool last_fused = false;  // the last sparsify call on this workspace ran the fused kernel
 };
 
 // host side (gk_host.cu)
@@ -82,6 +90,11 @@ void note_launch(int n = 1);
 // Stage timing: mark(ws, st, i) records event i (0 = before the first kernel) when tracing is on.
 void stage_mark(Workspace* ws, cudaStream_t st, int i);
 int64_t output_capacity(int64_t d);
+int selected_path();  // 0: fused kernel when usable, 1: three kernels with look-back
+int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                     float* val_out, int64_t* nnz_out, cudaStream_t st);
+int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                        float* val_out, int64_t* nnz_out, cudaStream_t st);
 
 inline int64_t num_compact_tiles(int64_t d) {
     return (d + kCompactTileElems - 1) / kCompactTileElems;
@@ -106,6 +119,12 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 // Streaming 128-bit load: the line is not expected to be read again.
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 __device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
     unsigned long long v;

@@ -1,0 +1,670 @@
+// gk_sparsify as ONE persistent cooperative kernel (Eq. 2 and Algorithm 1 of
+// arXiv 1911.08772).
+//
+// One CTA per SM owns a contiguous run of the vector and streams through it in
+// rows of 1024 float4 (16 KB; thread t takes float4 t of the row).  The three
+// phases of the method are separated by two grid barriers, and what fits of u
+// stays on chip between them:
+//
+//   phase A  u = g + eps, written over eps; the first rows are also kept in
+//            shared memory; fp64 partial sums per CTA; per (row, warp) the
+//            largest magnitude goes to a small table in shared memory.
+//   barrier  every CTA adds the partials in the same fixed order and forms
+//            mu, sigma, thres0 and the ten candidate thresholds for itself.
+//   phase B  counts of |u| > candidate for all ten candidates, from the
+//            on-chip copy where there is one, else from eps (L2 / HBM).
+//   barrier  every CTA reads all CTAs' counts, replays the rounds of
+//            Algorithm 1, and -- the count for the chosen threshold being
+//            known per CTA -- gets the output offset of its run directly.
+//            No look-back, no waiting between CTAs.
+//   phase C  groups of eight rows: a (row, warp) segment is read again only if
+//            its recorded maximum can exceed the threshold; an in-CTA scan
+//            orders the survivors; they are written as (index, value) pairs
+//            and their slots cleared.
+//
+// HBM traffic: 12 d bytes for phase A, 4 d for phase B on the rows that are not
+// on chip, and next to nothing for phase C (survivors are rare, so few segments
+// qualify).
+//
+// The barriers are counters in the workspace.  Every wait is bounded; a CTA
+// whose wait runs out records GK_DEV_TIMEOUT and leaves.  The kernel is
+// launched cooperatively, so all CTAs are resident and the waits do end.
+#include <math.h>
+
+#include "gk_alg1.cuh"
+#include "gk_common.cuh"
+
+namespace gk {
+
+constexpr int kFusedThreads = 1024;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kRowF4 = kFusedThreads;                  // float4 per row
+constexpr int kRowBytes = kRowF4 * 16;                 // 16 KB
+constexpr int kFusedSmemBytes = 13 * kRowBytes;        // dynamic shared memory: cache rows + table
+constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
+constexpr int kTableMaxRows = 384;                     // rows beyond this are ordered in groups and always re-read
+constexpr int kGroupRows = 8;                          // rows ordered by one in-CTA scan
+constexpr int kFusedMaxGrid = kFusedGridCap;
+constexpr int kBarrierPollLimit = 1 << 24;
+
+struct FusedShared {
+    double2 red[kFusedWarps];
+    unsigned int cta_counts[kNumCand];
+    unsigned long long col[kNumCand];   // counts over the whole vector
+    unsigned long long colpre[kNumCand];  // counts over the runs of the CTAs before this one
+    double cand64[kNumCand];
+    float cand32[kNumCand];
+    int order[kNumCand];                // candidate indices, ascending by threshold
+    float thr_sel;
+    int chosen;
+    int ok;
+    unsigned long long base;            // survivors in earlier CTAs
+    gk_stats stats;
+    // ordering scan of one group of rows
+    unsigned int wtot[kGroupRows][kFusedWarps];
+    unsigned int woff[kGroupRows][kFusedWarps];
+    unsigned int rtot[kGroupRows];
+    unsigned int rowpre[kTableMaxRows];  // survivors in the rows before each row of this CTA
+    unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
+};
+
+// Arrive at a barrier counter and wait until all G CTAs have arrived.
+// Returns false when the bounded wait ran out.
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int G, int* ok_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        int polls = 0;
+        bool ok = true;
+        while (true) {
+            unsigned int v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+            if (v >= G) break;
+            if (++polls > kBarrierPollLimit) { ok = false; break; }
+            __nanosleep(40);
+        }
+        *ok_flag = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *ok_flag != 0;
+}
+
+// 1.0f when a > c, else 0.0f: one compare instruction with a float result.
+__device__ __forceinline__ float gt_as_float(float a, float c) {
+    float r;
+    asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(c));
+    return r;
+}
+
+// Candidates LO..HI-1 (in ascending order of value) against the four magnitudes of one
+// float4.  The counters are floats: exact up to 2^24 per thread, far above a thread's share.
+template <int LO, int HI>
+__device__ __forceinline__ void count_tier(const float a0, const float a1, const float a2, const float a3,
+                                           const float (&cs)[kNumCand], float (&acc)[kNumCand]) {
+#pragma unroll
+    for (int j = LO; j < HI; ++j)
+        acc[j] += (gt_as_float(a0, cs[j]) + gt_as_float(a1, cs[j])) + (gt_as_float(a2, cs[j]) + gt_as_float(a3, cs[j]));
+}
+
+// rm: the segment's largest magnitude (top 16 bits, rounded up).  A candidate whose top 16
+// bits (rounded down) are not below rm cannot be exceeded by any element of the segment.
+__device__ __forceinline__ void count_float4(const float4 v, const unsigned int rm, const float (&cs)[kNumCand],
+                                             const unsigned int t5, const unsigned int t7,
+                                             float (&acc)[kNumCand]) {
+    const float a0 = fabsf(v.x), a1 = fabsf(v.y), a2 = fabsf(v.z), a3 = fabsf(v.w);
+    count_tier<0, 5>(a0, a1, a2, a3, cs, acc);
+    if (rm > t5) {  // warp-uniform
+        count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
+        if (rm > t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
+    }
+}
+
+__device__ __forceinline__ unsigned int max_mag_bits(const float4 u) {
+    return __float_as_uint(fmaxf(fmaxf(fabsf(u.x), fabsf(u.y)), fmaxf(fabsf(u.z), fabsf(u.w))));
+}
+
+__device__ __forceinline__ unsigned int mask_above(const float4 v, const float thr) {
+    return (unsigned)(fabsf(v.x) > thr) | ((unsigned)(fabsf(v.y) > thr) << 1) |
+           ((unsigned)(fabsf(v.z) > thr) << 2) | ((unsigned)(fabsf(v.w) > thr) << 3);
+}
+
+// rows_per_cta: rows of the run of every CTA; cache_rows: rows kept in shared
+// memory; table_rows: rows that have an entry in the maximum table.
+__global__ void __launch_bounds__(kFusedThreads, 1)
+k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
+           int rows_per_cta, int cache_rows, int table_rows, Ctrl* __restrict__ ctrl,
+           double2* __restrict__ partials, unsigned int* __restrict__ cta_counts,
+           unsigned int* __restrict__ bars, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+           int64_t* __restrict__ nnz_out, int64_t cap) {
+    extern __shared__ float4 cache[];  // cache_rows x kRowF4, then the table
+    __shared__ FusedShared sh;
+    unsigned short* table = reinterpret_cast<unsigned short*>(cache + (size_t)cache_rows * kRowF4);
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int c = blockIdx.x, G = gridDim.x;
+    const int64_t n4 = d >> 2;
+
+    // this CTA's run of float4
+    int64_t lo4 = (int64_t)c * rows_per_cta * kRowF4, hi4 = lo4 + (int64_t)rows_per_cta * kRowF4;
+    if (lo4 > n4) lo4 = n4;
+    if (hi4 > n4) hi4 = n4;
+    const int nrows = (int)((hi4 - lo4 + kRowF4 - 1) / kRowF4);
+    const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
+    const int64_t tail_i = (n4 << 2) + lane;
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    float4* e4 = reinterpret_cast<float4*>(eps);
+    float tail_u = 0.f;
+    if (c == 0 && tid == 0) {
+        ctrl->stats.status = GK_DEV_OK;
+        ctrl->phase_t[0] = global_timer_ns();
+    }
+
+    // ------------------------------------------------------------------ phase A
+    {
+        const double pv = (double)g[0];
+        double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
+        for (int r = 0; r < nrows; r += 2) {
+            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid, j = i + kRowF4;
+            const bool one = i < hi4, two = j < hi4;
+            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), b0 = a0, a1 = a0, b1 = a0;
+            if (one) { a0 = ld_stream(g4 + i); b0 = ld_stream(e4 + i); }
+            if (two) { a1 = ld_stream(g4 + j); b1 = ld_stream(e4 + j); }
+            const float4 u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
+            const float4 u1 = make_float4(a1.x + b1.x, a1.y + b1.y, a1.z + b1.z, a1.w + b1.w);
+            if (one) {
+                e4[i] = u0;
+                if (r < cache_rows) cache[(size_t)r * kRowF4 + tid] = u0;
+                const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
+                             x3 = (double)u0.w - pv;
+                s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
+                s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
+            }
+            if (two) {
+                e4[j] = u1;
+                if (r + 1 < cache_rows) cache[(size_t)(r + 1) * kRowF4 + tid] = u1;
+                const double x0 = (double)u1.x - pv, x1 = (double)u1.y - pv, x2 = (double)u1.z - pv,
+                             x3 = (double)u1.w - pv;
+                s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
+                s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
+            }
+            // largest magnitude of each (row, warp) segment, top 16 bits rounded up
+            const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
+            const unsigned int m1 = __reduce_max_sync(0xffffffffu, two ? max_mag_bits(u1) : 0u);
+            if (lane == 0) {
+                if (r < table_rows) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
+                if (r + 1 < table_rows && r + 1 < nrows)
+                    table[(r + 1) * kFusedWarps + w] = (unsigned short)((m1 + 0xffffu) >> 16);
+            }
+        }
+        if (owns_tail) {
+            tail_u = g[tail_i] + eps[tail_i];
+            eps[tail_i] = tail_u;
+            const double x = (double)tail_u - pv;
+            s0 += x; q0 = fma(x, x, q0);
+        }
+        const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
+        if (tid == 0) partials[c] = part;
+        if (!grid_barrier(&bars[0], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        // every CTA forms the same totals: thread t takes partial t, t + T, ...
+        double s = 0.0, q = 0.0;
+        for (int i = tid; i < G; i += kFusedThreads) {
+            const double2 p = __ldcg(&partials[i]);
+            s += p.x; q += p.y;
+        }
+        const double2 tot = block_sum2<kFusedThreads>(s, q, sh.red);
+        if (tid == 0) {
+            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
+            alg1_thresholds(st, tot.x, tot.y, pv, d, k, z);
+            // candidate indices in ascending order of threshold (insertion sort, ten entries)
+            for (int j = 0; j < kNumCand; ++j) {
+                int p = j;
+                while (p > 0 && sh.cand32[sh.order[p - 1]] > sh.cand32[j]) { sh.order[p] = sh.order[p - 1]; --p; }
+                sh.order[p] = j;
+            }
+        }
+        if (tid < kNumCand) sh.cta_counts[tid] = 0u;
+        if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
+        __syncthreads();
+    }
+
+    // ------------------------------------------------------------------ phase B
+    {
+        // candidates in ascending order of value; cs[j] = value, sh.order[j] = its index
+        float cs[kNumCand], acc[kNumCand];
+#pragma unroll
+        for (int j = 0; j < kNumCand; ++j) { cs[j] = sh.cand32[sh.order[j]]; acc[j] = 0.f; }
+        // tiers: candidates 5..6 and 7..9 are evaluated only for segments whose maximum can pass
+        const unsigned int t5 = cs[5] < 0.f ? 0u : (__float_as_uint(cs[5]) >> 16);
+        const unsigned int t7 = cs[7] < 0.f ? 0u : (__float_as_uint(cs[7]) >> 16);
+        const unsigned int always = 0x10000u;  // above every 16-bit maximum
+        const bool neg5 = cs[5] < 0.f, neg7 = cs[7] < 0.f;
+        int r = 0;
+        for (; r < nrows && r < cache_rows; ++r) {
+            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
+            if (neg5 || neg7) rm = always;
+            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
+                count_float4(cache[(size_t)r * kRowF4 + tid], rm, cs, t5, t7, acc);
+        }
+        for (; r < nrows; r += 4) {
+            float4 v[4];
+            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                v[q] = (i + q * kRowF4 < hi4) ? __ldcg(e4 + i + q * kRowF4) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                unsigned int rm = (r + q < table_rows) ? table[(r + q) * kFusedWarps + w] : always;
+                if (neg5 || neg7) rm = always;
+                if (i + q * kRowF4 < hi4) count_float4(v[q], rm, cs, t5, t7, acc);
+            }
+        }
+        if (owns_tail) {
+            const float a = fabsf(tail_u);
+#pragma unroll
+            for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < kNumCand; ++j) {
+            const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+            if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
+        }
+        __syncthreads();
+        if (tid < kNumCand) cta_counts[(size_t)c * kNumCand + tid] = sh.cta_counts[tid];
+        if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
+        if (!grid_barrier(&bars[1], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
+    }
+
+    // ------------------------------------------------------------------ resolve
+    {
+        // warp j adds column j over all CTAs and, separately, over the CTAs before this one
+        // (integer sums: the order does not matter); the loads are independent of each other
+        if (w < kNumCand) {
+            unsigned int v[kFusedMaxGrid / 32];
+#pragma unroll
+            for (int q = 0; q < kFusedMaxGrid / 32; ++q) {
+                const int t = lane + 32 * q;
+                v[q] = (t < G) ? __ldcg(&cta_counts[(size_t)t * kNumCand + w]) : 0u;
+            }
+            unsigned long long s = 0ull, pre = 0ull;
+#pragma unroll
+            for (int q = 0; q < kFusedMaxGrid / 32; ++q) {
+                s += v[q];
+                if (lane + 32 * q < c) pre += v[q];
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                s += __shfl_xor_sync(0xffffffffu, s, o);
+                pre += __shfl_xor_sync(0xffffffffu, pre, o);
+            }
+            if (lane == 0) { sh.col[w] = s; sh.colpre[w] = pre; }
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
+            sh.chosen = alg1_resolve(st, k);
+            sh.base = sh.colpre[sh.chosen];
+        }
+        __syncthreads();
+        if (c == 0 && tid == 0) {
+            const long long all = sh.stats.nnz;
+            const long long written = all < cap ? all : cap;
+            sh.stats.emitted = written;
+            if (all > cap) sh.stats.status |= GK_DEV_TRUNCATED;
+            const int late = ctrl->stats.status & GK_DEV_TIMEOUT;
+            ctrl->stats = sh.stats;
+            if (late) atomicOr(&ctrl->stats.status, late);
+            *nnz_out = written;
+            ctrl->phase_t[4] = global_timer_ns();
+        }
+        __syncthreads();
+    }
+
+    // ------------------------------------------------------------------ phase C
+    {
+        const float thr = sh.thr_sel;
+        const unsigned int mine = sh.cta_counts[sh.chosen];  // survivors in this CTA's run
+        // a segment can hold a survivor only if its recorded maximum (rounded up to 16 bits)
+        // exceeds the threshold's top 16 bits; a negative threshold admits everything
+        const bool all_pass = thr < 0.0f;
+        const unsigned int thr16 = __float_as_uint(fmaxf(thr, 0.0f)) >> 16;
+        unsigned long long run = sh.base;
+        const int trows = nrows < table_rows ? nrows : table_rows;  // rows covered by the table
+        if (mine != 0u) {
+            // step 1: every warp counts the survivors of its qualifying segments; the table
+            // entry of a segment is replaced by that count (0 where it cannot qualify).
+            // Qualifying rows are gathered eight at a time so that their loads overlap.
+            constexpr unsigned short kPending = 0xffffu;
+            for (int r = lane; r < trows; r += 32) {
+                const bool ql = all_pass || table[r * kFusedWarps + w] > thr16;
+                table[r * kFusedWarps + w] = ql ? kPending : (unsigned short)0;
+            }
+            __syncwarp();
+            // up to kGroupRows rows of this warp whose entry satisfies want(entry), from `cursor` on
+            auto gather = [&](int& cursor, const bool want_pending) -> int {
+                int n = 0;
+                while (n < kGroupRows && cursor < trows) {
+                    const int r = cursor + lane;
+                    unsigned int e = 0u;
+                    if (r < trows) e = table[r * kFusedWarps + w];
+                    const bool hit = want_pending ? (e == kPending) : (e != 0u);
+                    unsigned int b = __ballot_sync(0xffffffffu, hit);
+                    while (b && n < kGroupRows) {
+                        const int bit = __ffs(b) - 1;
+                        if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
+                        ++n;
+                        b &= b - 1u;
+                    }
+                    if (b) { cursor += __ffs(b) - 1; break; }
+                    cursor += 32;
+                }
+                __syncwarp();
+                return n;
+            };
+            for (int cursor = 0; cursor < trows;) {
+                const int n = gather(cursor, true);
+                float4 v[kGroupRows];
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < n) {
+                        const int r = sh.qrow[w][q];
+                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                        if (i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    if (q < n) {
+                        const int r = sh.qrow[w][q];
+                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                        const unsigned int cnt =
+                            __reduce_add_sync(0xffffffffu, i < hi4 ? __popc(mask_above(v[q], thr)) : 0u);
+                        if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
+                    }
+                }
+                __syncwarp();
+            }
+            __syncthreads();
+            // step 2: survivors per row, exclusive scan over the rows (thread t takes row t)
+            {
+                unsigned int mine_row = 0u;
+                if (tid < trows) {
+                    const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
+#pragma unroll
+                    for (int q = 0; q < kTableRowBytes / 16; ++q) {
+                        const uint4 x = tv[q];
+                        mine_row += (x.x & 0xffffu) + (x.x >> 16) + (x.y & 0xffffu) + (x.y >> 16) +
+                                    (x.z & 0xffffu) + (x.z >> 16) + (x.w & 0xffffu) + (x.w >> 16);
+                    }
+                }
+                unsigned int s = mine_row;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int t = __shfl_up_sync(0xffffffffu, s, o);
+                    if (lane >= o) s += t;
+                }
+                if (lane == 31) sh.wtot[0][w] = s;
+                __syncthreads();
+                if (w == 0) {
+                    const unsigned int x = sh.wtot[0][lane];
+                    unsigned int y = x;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned int t = __shfl_up_sync(0xffffffffu, y, o);
+                        if (lane >= o) y += t;
+                    }
+                    sh.woff[0][lane] = y - x;
+                    if (lane == 31) sh.rtot[0] = y;
+                }
+                __syncthreads();
+                if (tid < trows) sh.rowpre[tid] = sh.woff[0][w] + s - mine_row;
+                __syncthreads();
+            }
+            // step 3: every warp writes the survivors of its segments that have any
+            for (int cursor = 0; cursor < trows;) {
+                const int n = gather(cursor, false);
+                float4 v[kGroupRows];
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < n) {
+                        const int r = sh.qrow[w][q];
+                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                        if (i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    if (q >= n) continue;
+                    const int r = sh.qrow[w][q];
+                    const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                    const unsigned int m = i < hi4 ? mask_above(v[q], thr) : 0u;
+                    // survivors of this row in the warps before this one
+                    const unsigned int before =
+                        __reduce_add_sync(0xffffffffu, lane < w ? (unsigned int)table[r * kFusedWarps + lane] : 0u);
+                    const unsigned int c_m = __popc(m);
+                    unsigned int sc = c_m;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned int t = __shfl_up_sync(0xffffffffu, sc, o);
+                        if (lane >= o) sc += t;
+                    }
+                    if (m) {
+                        unsigned long long p = run + sh.rowpre[r] + before + (sc - c_m);
+                        const int64_t e0 = i << 2;
+                        const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            if (m & (1u << t)) {
+                                if ((long long)p < cap) {
+                                    idx_out[p] = (int32_t)(e0 + t);
+                                    val_out[p] = vv[t];
+                                    eps[e0 + t] = 0.0f;
+                                }
+                                ++p;
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            run += sh.rtot[0];
+            __syncthreads();  // the scan arrays are reused below
+            // rows beyond the table (vectors of more than ~230 M elements): ordered in groups
+            for (int r0 = trows; r0 < nrows; r0 += kGroupRows) {
+                // does any segment of this group qualify?  (the same answer in every warp)
+                bool any = all_pass;
+                if (!any) {
+#pragma unroll
+                    for (int q = 0; q < kGroupRows; ++q) {
+                        const int r = r0 + q;
+                        if (r < nrows) any |= (r >= table_rows) || (table[r * kFusedWarps + lane] > thr16);
+                    }
+                    any = __any_sync(0xffffffffu, any);
+                }
+                if (!any) continue;
+                float4 v[kGroupRows];
+                unsigned int m[kGroupRows];
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    const int r = r0 + q;
+                    const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    m[q] = 0u;
+                    // warp-uniform: skip the segment when its maximum cannot pass
+                    const bool look = r < nrows &&
+                                      (all_pass || r >= table_rows || table[r * kFusedWarps + w] > thr16);
+                    if (look && i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                }
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    const int64_t i = lo4 + (int64_t)(r0 + q) * kRowF4 + tid;
+                    if (r0 + q < nrows && i < hi4) m[q] = mask_above(v[q], thr);
+                }
+                // order: (row, warp, lane).  Packed byte scans inside the warp, then over warps.
+                unsigned int incl[kGroupRows / 4];
+#pragma unroll
+                for (int h = 0; h < kGroupRows / 4; ++h) {
+                    unsigned int p = __popc(m[4 * h]) | (__popc(m[4 * h + 1]) << 8) | (__popc(m[4 * h + 2]) << 16) |
+                                     (__popc(m[4 * h + 3]) << 24);
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned int t = __shfl_up_sync(0xffffffffu, p, o);
+                        if (lane >= o) p += t;  // bytes hold at most 32 * 4 = 128
+                    }
+                    incl[h] = p;
+                    if (lane == 31) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) sh.wtot[4 * h + q][w] = (p >> (8 * q)) & 0xffu;
+                    }
+                }
+                __syncthreads();
+                if (w < kGroupRows) {
+                    const unsigned int x = sh.wtot[w][lane];
+                    unsigned int s = x;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned int t = __shfl_up_sync(0xffffffffu, s, o);
+                        if (lane >= o) s += t;
+                    }
+                    sh.woff[w][lane] = s - x;
+                    if (lane == 31) sh.rtot[w] = s;
+                }
+                __syncthreads();
+                unsigned long long row_base = run;
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    if (m[q]) {
+                        const unsigned int c_q = __popc(m[q]);
+                        unsigned long long p = row_base + sh.woff[q][w] + ((incl[q >> 2] >> (8 * (q & 3))) & 0xffu) - c_q;
+                        const int64_t e0 = (lo4 + (int64_t)(r0 + q) * kRowF4 + tid) << 2;
+                        const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            if (m[q] & (1u << t)) {
+                                if ((long long)p < cap) {
+                                    idx_out[p] = (int32_t)(e0 + t);
+                                    val_out[p] = vv[t];
+                                    eps[e0 + t] = 0.0f;
+                                }
+                                ++p;
+                            }
+                        }
+                    }
+                    row_base += sh.rtot[q];
+                }
+                run = row_base;
+                __syncthreads();  // the scan arrays are reused by the next group
+            }
+        }
+        // the ragged tail comes last in index order
+        if ((c == G - 1) && (w == kFusedWarps - 1) && (d & 3)) {
+            const bool hit = owns_tail && (fabsf(tail_u) > thr);
+            const unsigned int bal = __ballot_sync(0xffffffffu, hit);
+            if (hit) {
+                const unsigned long long p = run + __popc(bal & ((1u << lane) - 1u));
+                if ((long long)p < cap) {
+                    idx_out[p] = (int32_t)tail_i;
+                    val_out[p] = tail_u;
+                    eps[tail_i] = 0.0f;
+                }
+            }
+        }
+    }
+
+    if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
+
+leave:
+    // the CTA that leaves last clears the barrier counters for the next call
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(&bars[2], 1u);
+        if (t == (unsigned)G - 1) {
+            ctrl->phase_t[6] = global_timer_ns();
+            bars[0] = 0u; bars[1] = 0u;
+            __threadfence();
+            bars[2] = 0u;
+        }
+    }
+}
+
+// Host side -----------------------------------------------------------------
+struct FusedPlan {
+    bool ready = false, usable = false;
+    int grid = 0;
+};
+static FusedPlan g_plan[64];
+
+static FusedPlan* fused_plan(int dev, int sm_count) {
+    if (dev < 0 || dev >= 64) return nullptr;
+    FusedPlan& p = g_plan[dev];
+    if (p.ready) return &p;
+    p.ready = true;
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return &p;
+    if (cudaFuncSetAttribute(k_gk_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBytes) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return &p;
+    }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused, kFusedThreads, kFusedSmemBytes) !=
+            cudaSuccess || occ < 1) {
+        cudaGetLastError();
+        return &p;
+    }
+    p.grid = sm_count < kFusedMaxGrid ? sm_count : kFusedMaxGrid;
+    p.usable = true;
+    return &p;
+}
+
+// Returns GK_OK when the fused kernel was enqueued, 1 when it cannot be used on
+// this device or for this call (the caller then takes the three-kernel path),
+// or an error.
+int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                     float* val_out, int64_t* nnz_out, cudaStream_t st) {
+    int dev = 0;
+    GK_CUDA_TRY(cudaGetDevice(&dev));
+    FusedPlan* p = fused_plan(dev, ws->sm_count);
+    if (!p || !p->usable || k >= d) return 1;
+    const int64_t n4 = d >> 2;
+    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;  // rows in the whole vector
+    int64_t G = p->grid;
+    int64_t rows_per_cta = (n_rows + G - 1) / G;
+    if (rows_per_cta < 1) rows_per_cta = 1;
+    G = (n_rows + rows_per_cta - 1) / rows_per_cta;  // no CTA without rows
+    if (G < 1) G = 1;
+    int rpc = (int)rows_per_cta;
+    // shared memory: the maximum table first claims its share, the rest caches rows
+    int table_rows = rpc < kTableMaxRows ? rpc : kTableMaxRows;
+    const int table_bytes = (table_rows * kTableRowBytes + 15) / 16 * 16;
+    int cache_rows = (kFusedSmemBytes - table_bytes) / kRowBytes;
+    if (cache_rows > rpc) cache_rows = rpc;
+    const double pq = 1.0 - (double)k / (double)d;  // Algorithm 1: p = 1 - k/d
+    double z = normal_quantile_upper(1.0 - pq);
+    int64_t cap = output_capacity(d);
+    Ctrl* ctrl = ws->ctrl;
+    double2* partials = ws->partials;
+    unsigned int* cta_counts = ws->cta_counts;
+    unsigned int* bars = ws->bars;
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&cache_rows,
+                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
+                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
+    stage_mark(ws, st, 0);
+    GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
+                                            (size_t)kFusedSmemBytes, st));
+    note_launch();
+    stage_mark(ws, st, 1);
+    ws->last_fused = true;
+    return GK_OK;
+}
+
+}  // namespace gk

@@ -49,7 +49,7 @@ int64_t output_capacity(int64_t d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t ctrl, partials, hist, tile_status, seg, total;
+    size_t ctrl, partials, hist, cta_counts, bars, tile_status, seg, total;
 };
 
 static Layout layout_for(int64_t d, int32_t S) {
@@ -58,6 +58,8 @@ static Layout layout_for(int64_t d, int32_t S) {
     L.ctrl = at;        at = align_up(at + sizeof(Ctrl), 256);
     L.partials = at;    at = align_up(at + sizeof(double2) * kMaxPartials, 256);
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
+    L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
+    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 4, 256);
     L.tile_status = at; at = align_up(at + sizeof(unsigned long long) * (size_t)num_compact_tiles(d), 256);
     L.seg = at;         at = align_up(at + segmented_scratch_bytes(d, S), 256);
     L.total = at;
@@ -92,6 +94,8 @@ int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out
         ws.ctrl = reinterpret_cast<Ctrl*>(b + L.ctrl);
         ws.partials = reinterpret_cast<double2*>(b + L.partials);
         ws.hist = reinterpret_cast<unsigned int*>(b + L.hist);
+        ws.cta_counts = reinterpret_cast<unsigned int*>(b + L.cta_counts);
+        ws.bars = reinterpret_cast<unsigned int*>(b + L.bars);
         ws.tile_status = reinterpret_cast<unsigned long long*>(b + L.tile_status);
         ws.seg_block = b + L.seg;
         GK_CUDA_TRY(cudaDeviceGetAttribute(&ws.sm_count, cudaDevAttrMultiProcessorCount, dev));
@@ -115,8 +119,8 @@ struct HostStage {
 };
 static std::map<int, HostStage> g_stage;
 
-int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
-                        int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st);
+static std::atomic<int> g_path{0};
+int selected_path() { return g_path.load(std::memory_order_relaxed); }
 
 }  // namespace gk
 
@@ -125,6 +129,12 @@ using namespace gk;
 extern "C" int gk_set_capacity(int64_t cap) {
     if (cap < 0) return GK_ERR_CAPACITY;
     g_capacity.store(cap);
+    return GK_OK;
+}
+
+extern "C" int gk_set_path(int path) {
+    if (path < 0 || path > 1) return GK_ERR_SIZE;
+    g_path.store(path);
     return GK_OK;
 }
 
@@ -178,6 +188,13 @@ extern "C" int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages
     *n_stages = ws->n_stages;
     for (int i = 0; i < ws->n_stages; ++i)
         GK_CUDA_TRY(cudaEventElapsedTime(&ms_out[i], ws->ev[i], ws->ev[i + 1]));
+    if (ws->last_fused && ws->n_stages == 1) {
+        // one kernel: after its event time, the three phases from the kernel's own timestamps
+        unsigned long long t[8];
+        GK_CUDA_TRY(cudaMemcpy(t, ws->ctrl->phase_t, sizeof(t), cudaMemcpyDeviceToHost));
+        for (int i = 0; i < 6; ++i) ms_out[1 + i] = (float)((double)(t[i + 1] - t[i]) * 1e-6);
+        *n_stages = 7;
+    }
     return GK_OK;
 }
 

@@ -199,8 +199,8 @@ static int reduction_grid(const Workspace* ws, int64_t d, int threads, int unrol
     return (int)(want < cap ? want : cap);
 }
 
-// Enqueue the three kernels on an already validated call.
-int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
+// Enqueue the three-kernel (look-back) path on an already validated call.
+int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
                         int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st) {
     const int n_tiles = (int)num_compact_tiles(d);
     double z = -INFINITY;
@@ -225,8 +225,20 @@ int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, in
         nullptr);
     note_launch();
     stage_mark(ws, st, 3);
+    ws->last_fused = false;
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;
+}
+
+// Enqueue one step by the selected path: the fused cooperative kernel unless it
+// cannot be used on this device (or for this call), else the three-kernel path.
+int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
+                        int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st) {
+    if (selected_path() != 1) {
+        const int rc = enqueue_gk_fused(ws, g, eps, d, k, idx_out, val_out, nnz_out, st);
+        if (rc != 1) return rc;
+    }
+    return enqueue_gk_three_kernel(ws, g, eps, d, k, idx_out, val_out, nnz_out, st);
 }
 
 }  // namespace gk

@@ -26,13 +26,21 @@ def _library():
     yield
 
 
+@pytest.fixture(params=[0, 1], ids=["fused", "three_kernel"])
+def gk_path(request):
+    """Run a test once per implementation of gk_sparsify."""
+    gk.gk_set_path(request.param)
+    yield request.param
+    gk.gk_set_path(0)
+
+
 # ------------------------------------------------------------------ small sizes, every boundary
 SMALL_D = [1, 2, 3, 4, 5, 7, 8, 31, 32, 33, 127, 128, 129, 1023, 1024, 1025, 4095, 4096, 4097,
            TILE - 1, TILE, TILE + 1, 2 * TILE + 3, 5 * TILE - 2, 100_003]
 
 
 @pytest.mark.parametrize("d", SMALL_D)
-def test_gk_sparsify_small_sizes(d):
+def test_gk_sparsify_small_sizes(d, gk_path):
     rng = wl.misc_rng(1000 + d)
     g = (rng.standard_normal(d) * 1e-3).astype(np.float32)
     e = (rng.standard_normal(d) * 2e-3).astype(np.float32)
@@ -41,7 +49,7 @@ def test_gk_sparsify_small_sizes(d):
         check_gk_step(step, g, e, k)
 
 
-def test_gk_sparsify_special_values():
+def test_gk_sparsify_special_values(gk_path):
     d = 3 * TILE + 1
     rng = wl.misc_rng(7)
     g = (rng.standard_normal(d) * 1e-3).astype(np.float32)
@@ -66,7 +74,7 @@ def test_gk_sparsify_special_values():
     assert st.nnz == d
 
 
-def test_gk_hand_built_branch_cases():
+def test_gk_hand_built_branch_cases(gk_path):
     # the same level vectors that pin the oracle's branch sequences
     from test_oracle_pins import _branch_cases, _levels_vector
     for name, d, k, levels, rounds, counts, fn, fd, nnz in _branch_cases():
@@ -77,7 +85,7 @@ def test_gk_hand_built_branch_cases():
         assert abs(st.thr_final / st.thres0 - fn / fd) < 1e-15
 
 
-def test_gk_capacity_truncation():
+def test_gk_capacity_truncation(gk_path):
     d = 4 * TILE + 5
     u = wl.normal(d, 1.0, step=2)
     z = np.zeros(d, dtype=np.float32)
@@ -90,7 +98,7 @@ def test_gk_capacity_truncation():
         gk.gk_set_capacity(0)
 
 
-def test_gk_is_deterministic_and_stateless():
+def test_gk_is_deterministic_and_stateless(gk_path):
     d = 1_000_003
     g = wl.laplace_mixture(d, step=3)
     e = wl.normal(d, 1e-4, step=4)
@@ -103,7 +111,7 @@ def test_gk_is_deterministic_and_stateless():
         assert np.array_equal(o[0], outs[0][0]) and o[1:] == outs[0][1:]
 
 
-def test_gk_on_a_side_stream():
+def test_gk_on_a_side_stream(gk_path):
     d = 300_007
     g = wl.normal(d, 1e-3, step=11)
     z = np.zeros(d, np.float32)
@@ -225,7 +233,7 @@ def _ec_loop(w, rho, steps, check_every=1, also=None):
     return eps
 
 
-def test_workload_resnet20_normal():
+def test_workload_resnet20_normal(gk_path):
     w = wl.resnet20_normal()
     assert w.k("1e-3") == 270
     _ec_loop(w, "1e-3", 1 + 10)
@@ -236,6 +244,32 @@ def test_workload_vgg16_laplace_mixture_100_steps():
     nnzs = []
     _ec_loop(w, "1e-3", 100, also=lambda t, st: nnzs.append(st.nnz))
     assert min(nnzs) > 0
+
+
+def test_workload_resnet50_three_kernel_path():
+    gk.gk_set_path(1)
+    try:
+        _ec_loop(wl.resnet50_segmented(), "1e-3", 5)
+    finally:
+        gk.gk_set_path(0)
+
+
+def test_both_paths_agree_bit_for_bit():
+    w = wl.vgg16_laplace_mixture()
+    g = w.grad(0, None)
+    e = wl.normal(w.d, 1e-4, step=9)
+    k = w.k("1e-3")
+    step = DeviceStep(w.d)
+    outs = []
+    for path in (0, 1):
+        gk.gk_set_path(path)
+        try:
+            eps_new, st = check_gk_step(step, g, e, k)
+        finally:
+            gk.gk_set_path(0)
+        outs.append((bits(eps_new).copy(), st.thr_final, st.counts, st.nnz))
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][2:] == outs[1][2:]
+    assert abs(outs[0][1] / outs[1][1] - 1) < 1e-12
 
 
 @pytest.mark.parametrize("rho", ["1e-3", "1e-2"])
