@@ -149,6 +149,33 @@ int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx
 int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                      float* val_out, int64_t* nnz_out, gk_stats* stats_out);
 
+/*
+ * gk_sparsify_static -- gk_sparsify for callers that must not allocate device
+ * memory (the paper has no counterpart: this is a deployment variant of the
+ * same step, not another method).  Think of a step that runs under a framework
+ * allocator with a fixed budget, or of a service that bans cudaMalloc once it
+ * is serving because that call stalls the whole device.  Same arguments, same
+ * results and same capacity rule as gk_sparsify, but the call never reaches
+ * cudaMalloc, cudaFree or any routine that allocates: its scratch is a fixed
+ * 32 KB array inside the library image, present on every GPU that loads the
+ * library for as long as the process lives.
+ *
+ * Limits: 1 <= k < d <= 2^31 - 1 (d beyond that returns GK_ERR_SIZE; k = d
+ * returns GK_ERR_K: selecting everything is left to gk_sparsify); the device
+ * must support cooperative launch and the launch must fit the array's 512
+ * per-CTA slots, else GK_ERR_LIMIT.
+ *
+ * The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress) and keeps it; make that first call before any stream
+ * capture begins.  All calls on a device share the one array, which keeps
+ * whatever the previous call left in it; the call clears the words that have
+ * to start at zero.  Two calls that overlap on the GPU (different streams)
+ * would race on the array: keep them in order.  There is no statistics record
+ * to read back for this call.
+ */
+int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                       float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
 /* Output capacity of idx_out / val_out for the sparsify calls, in pairs.
  * 0 (the default) means "d".  Process-wide; returns GK_ERR_CAPACITY if cap < 0. */
 int gk_set_capacity(int64_t cap);

@@ -21,7 +21,7 @@ GK_DEV_BAD_SEGMENTS = 4
 
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
-    "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
+    "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
 ]
 
@@ -71,6 +71,8 @@ def load() -> C.CDLL:
     L = C.CDLL(LIB_PATH)
     vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int32
     L.gk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.gk_sparsify_static.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.gk_sparsify_static.restype = C.c_int
     L.gk_sparsify_segmented.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.topk_exact.argtypes = [vp, i64, i64, vp, vp, vp]
     L.topk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
@@ -130,6 +132,16 @@ def gk_sparsify(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
     _check(load().gk_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), d, k,
                               _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
                               _dev(nnz_out, torch.int64), _stream()))
+
+
+def gk_sparsify_static(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
+    """gk_sparsify without any device allocation: the scratch is a fixed array inside the
+    library (see gk.h for who needs this and for the limits)."""
+    import torch
+    d = g.numel()
+    _check(load().gk_sparsify_static(_dev(g, torch.float32), _dev(eps, torch.float32), d, k,
+                                     _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
+                                     _dev(nnz_out, torch.int64), _stream()))
 
 
 def gk_sparsify_segmented(g, eps, seg_offsets, seg_k, idx_out, val_out, seg_nnz_out, nnz_out) -> None:

@@ -31,6 +31,8 @@
 // launched cooperatively, so all CTAs are resident and the waits do end.
 #include <math.h>
 
+#include <mutex>
+
 #include "gk_alg1.cuh"
 #include "gk_common.cuh"
 
@@ -668,3 +670,103 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
 }
 
 }  // namespace gk
+
+// ---------------------------------------------------------------------------
+// gk_sparsify_static: the same kernel for callers that must not allocate.
+//
+// Some callers cannot let a library call cudaMalloc on their behalf: code that
+// runs under a framework's caching allocator with a fixed memory budget, a
+// service that forbids device allocations after start-up because cudaMalloc
+// synchronises the whole device, or a step that has to behave the same on its
+// first and on its millionth call.  For them the scratch of the fused kernel
+// (control block, per-CTA partial sums, per-CTA candidate counts, barrier
+// counters) lives in the fixed array below instead of a workspace obtained
+// from cudaMalloc.  The array is part of the library image: every GPU that
+// loads the library holds these 32 KB until the process exits.
+// ---------------------------------------------------------------------------
+namespace gk {
+
+constexpr size_t kStaticCtrlBytes = (sizeof(Ctrl) + 255) / 256 * 256;
+constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap;                // 8 KB
+constexpr size_t kStaticCountBytes = sizeof(unsigned int) * kFusedGridCap * kNumCand;  // 20 KB
+constexpr size_t kStaticBarBytes = 256;
+constexpr size_t kStaticScratchBytes = 32 * 1024;
+static_assert(kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes + kStaticBarBytes <= kStaticScratchBytes,
+              "static scratch too small");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch per device.  In host code the name of a
+// __device__ array is only a handle for the runtime, not an address a kernel
+// can use; cudaGetSymbolAddress translates it for the device that is current.
+struct StaticScratch {
+    bool ready = false;
+    unsigned char* base = nullptr;
+    int sm_count = 0;
+};
+static StaticScratch g_static[64];
+static std::mutex g_static_mu;
+
+}  // namespace gk
+
+extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                                  float* val_out, int64_t* nnz_out, gk_stream_t stream) {
+    using namespace gk;
+    if (!g || !eps || !idx_out || !val_out || !nnz_out) return GK_ERR_NULL;
+    if (d < 1 || d > 2147483647ll) return GK_ERR_SIZE;
+    if (k < 1 || k >= d) return GK_ERR_K;  // k = d (select everything) is served by gk_sparsify only
+    if (((uintptr_t)g & 15u) || ((uintptr_t)eps & 15u)) return GK_ERR_ALIGN;
+    const uintptr_t ga = (uintptr_t)g, ea = (uintptr_t)eps, nb = (uintptr_t)d * 4u;
+    if (ga < ea + nb && ea < ga + nb) return GK_ERR_ALIAS;
+    cudaStream_t st = (cudaStream_t)stream;
+    int dev = 0;
+    GK_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return GK_ERR_LIMIT;
+    StaticScratch* ss = &g_static[dev];
+    {
+        // first call on this device: look the array's device address up once
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!ss->ready) {
+            void* p = nullptr;
+            GK_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+            GK_CUDA_TRY(cudaDeviceGetAttribute(&ss->sm_count, cudaDevAttrMultiProcessorCount, dev));
+            ss->base = static_cast<unsigned char*>(p);
+            ss->ready = true;
+        }
+    }
+    FusedPlan* plan = fused_plan(dev, ss->sm_count);
+    if (!plan || !plan->usable) return GK_ERR_LIMIT;  // no cooperative launch on this device
+
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(ss->base);
+    double2* partials = reinterpret_cast<double2*>(ss->base + kStaticCtrlBytes);
+    unsigned int* cta_counts = reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes);
+    unsigned int* bars =
+        reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes);
+
+    const int64_t n4 = d >> 2;
+    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;
+    int64_t G = plan->grid;
+    int64_t rows_per_cta = (n_rows + G - 1) / G;
+    if (rows_per_cta < 1) rows_per_cta = 1;
+    G = (n_rows + rows_per_cta - 1) / rows_per_cta;
+    if (G < 1) G = 1;
+    if (G > kFusedGridCap) return GK_ERR_LIMIT;  // more CTAs than the fixed array has slots for
+    // The array keeps what the last call left.  The barrier counters must start at zero; the
+    // kernel resets them when it ends, but a call that was cut short would not have.
+    GK_CUDA_TRY(cudaMemsetAsync(bars, 0, kStaticBarBytes, st));
+    int rpc = (int)rows_per_cta;
+    int table_rows = rpc < kTableMaxRows ? rpc : kTableMaxRows;
+    const int table_bytes = (table_rows * kTableRowBytes + 15) / 16 * 16;
+    int cache_rows = (kFusedSmemBytes - table_bytes) / kRowBytes;
+    if (cache_rows > rpc) cache_rows = rpc;
+    const double pq = 1.0 - (double)k / (double)d;
+    double z = normal_quantile_upper(1.0 - pq);
+    int64_t cap = output_capacity(d);
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&cache_rows,
+                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
+                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
+    GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
+                                            (size_t)kFusedSmemBytes, st));
+    note_launch();
+    return GK_OK;
+}
