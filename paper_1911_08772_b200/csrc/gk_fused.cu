@@ -6,9 +6,11 @@
 // phases of the method are separated by two grid barriers, and what fits of u
 // stays on chip between them:
 //
-//   phase A  u = g + eps, written over eps; the first rows are also kept in
-//            shared memory; fp64 partial sums per CTA; per (row, warp) the
-//            largest magnitude goes to a small table in shared memory.
+//   phase A  g and eps arrive through a ring of asynchronous copies (cp.async,
+//            three rows ahead); u = g + eps is written over eps and into the
+//            shared-memory slot its eps came through, so the last rows of the
+//            run are still on chip afterwards; fp64 partial sums per CTA; per
+//            (row, warp) the largest magnitude goes to a small table.
 //   barrier  every CTA adds the partials in the same fixed order and forms
 //            mu, sigma, thres0 and the ten candidate thresholds for itself.
 //   phase B  counts of |u| > candidate for all ten candidates, from the
@@ -42,7 +44,8 @@ constexpr int kFusedThreads = 1024;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kRowF4 = kFusedThreads;                  // float4 per row
 constexpr int kRowBytes = kRowF4 * 16;                 // 16 KB
-constexpr int kFusedSmemBytes = 13 * kRowBytes;        // dynamic shared memory: cache rows + table
+constexpr int kFusedSmemBytes = 13 * kRowBytes;        // dynamic shared memory: g ring, u slots, table
+constexpr int kStages = 4;                             // rows of g (and eps) in flight per CTA, plus one
 constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
 constexpr int kTableMaxRows = 384;                     // rows beyond this are ordered in groups and always re-read
 constexpr int kGroupRows = 8;                          // rows ordered by one in-CTA scan
@@ -70,6 +73,14 @@ struct FusedShared {
     unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
 };
 
+// 16-byte asynchronous copy global -> shared, bypassing L1.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const unsigned int s = (unsigned int)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 // Arrive at a barrier counter and wait until all G CTAs have arrived.
 // Returns false when the bounded wait ran out.
 __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int G, int* ok_flag) {
@@ -131,17 +142,21 @@ __device__ __forceinline__ unsigned int mask_above(const float4 v, const float t
            ((unsigned)(fabsf(v.z) > thr) << 2) | ((unsigned)(fabsf(v.w) > thr) << 3);
 }
 
-// rows_per_cta: rows of the run of every CTA; cache_rows: rows kept in shared
-// memory; table_rows: rows that have an entry in the maximum table.
+// rows_per_cta: rows of the run of every CTA; u_slots: row slots of shared memory
+// that receive eps and then hold u (the last u_slots rows of the run stay on
+// chip); table_rows: rows that have an entry in the maximum table.
+// Shared memory: [kStages rows of g in flight][u_slots rows][table].
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
-           int rows_per_cta, int cache_rows, int table_rows, Ctrl* __restrict__ ctrl,
+           int rows_per_cta, int u_slots, int table_rows, Ctrl* __restrict__ ctrl,
            double2* __restrict__ partials, unsigned int* __restrict__ cta_counts,
            unsigned int* __restrict__ bars, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
            int64_t* __restrict__ nnz_out, int64_t cap) {
-    extern __shared__ float4 cache[];  // cache_rows x kRowF4, then the table
+    extern __shared__ float4 smem4[];
     __shared__ FusedShared sh;
-    unsigned short* table = reinterpret_cast<unsigned short*>(cache + (size_t)cache_rows * kRowF4);
+    float4* gring = smem4;                                   // kStages x kRowF4
+    float4* uslot = smem4 + (size_t)kStages * kRowF4;        // u_slots x kRowF4
+    unsigned short* table = reinterpret_cast<unsigned short*>(uslot + (size_t)u_slots * kRowF4);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int c = blockIdx.x, G = gridDim.x;
     const int64_t n4 = d >> 2;
@@ -165,39 +180,40 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     {
         const double pv = (double)g[0];
         double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
-        for (int r = 0; r < nrows; r += 2) {
-            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid, j = i + kRowF4;
-            const bool one = i < hi4, two = j < hi4;
-            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), b0 = a0, a1 = a0, b1 = a0;
-            if (one) { a0 = ld_stream(g4 + i); b0 = ld_stream(e4 + i); }
-            if (two) { a1 = ld_stream(g4 + j); b1 = ld_stream(e4 + j); }
-            const float4 u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
-            const float4 u1 = make_float4(a1.x + b1.x, a1.y + b1.y, a1.z + b1.z, a1.w + b1.w);
+        // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
+        // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
+        auto fetch = [&](int r) {
+            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+            if (r < nrows && i < hi4) {
+                cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + i);
+                cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + i);
+            }
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int r = 0; r < kStages - 1; ++r) fetch(r);
+        for (int r = 0; r < nrows; ++r) {
+            fetch(r + kStages - 1);
+            cp_async_wait<kStages - 1>();
+            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+            const bool one = i < hi4;
+            float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one) {
+                float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
+                const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *us;
+                u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
                 e4[i] = u0;
-                if (r < cache_rows) cache[(size_t)r * kRowF4 + tid] = u0;
+                *us = u0;
                 const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
                              x3 = (double)u0.w - pv;
                 s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
                 s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
             }
-            if (two) {
-                e4[j] = u1;
-                if (r + 1 < cache_rows) cache[(size_t)(r + 1) * kRowF4 + tid] = u1;
-                const double x0 = (double)u1.x - pv, x1 = (double)u1.y - pv, x2 = (double)u1.z - pv,
-                             x3 = (double)u1.w - pv;
-                s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
-                s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
-            }
             // largest magnitude of each (row, warp) segment, top 16 bits rounded up
             const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
-            const unsigned int m1 = __reduce_max_sync(0xffffffffu, two ? max_mag_bits(u1) : 0u);
-            if (lane == 0) {
-                if (r < table_rows) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
-                if (r + 1 < table_rows && r + 1 < nrows)
-                    table[(r + 1) * kFusedWarps + w] = (unsigned short)((m1 + 0xffffu) >> 16);
-            }
+            if (lane == 0 && r < table_rows) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
         }
+        cp_async_wait<0>();
         if (owns_tail) {
             tail_u = g[tail_i] + eps[tail_i];
             eps[tail_i] = tail_u;
@@ -243,25 +259,27 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         const unsigned int t7 = cs[7] < 0.f ? 0u : (__float_as_uint(cs[7]) >> 16);
         const unsigned int always = 0x10000u;  // above every 16-bit maximum
         const bool neg5 = cs[5] < 0.f, neg7 = cs[7] < 0.f;
+        const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
         int r = 0;
-        for (; r < nrows && r < cache_rows; ++r) {
-            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
-            if (neg5 || neg7) rm = always;
-            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
-                count_float4(cache[(size_t)r * kRowF4 + tid], rm, cs, t5, t7, acc);
-        }
-        for (; r < nrows; r += 4) {
+        for (; r < first_kept; r += 4) {
             float4 v[4];
             const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-                v[q] = (i + q * kRowF4 < hi4) ? __ldcg(e4 + i + q * kRowF4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[q] = (r + q < first_kept && i + q * kRowF4 < hi4) ? __ldcg(e4 + i + q * kRowF4)
+                                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 unsigned int rm = (r + q < table_rows) ? table[(r + q) * kFusedWarps + w] : always;
                 if (neg5 || neg7) rm = always;
-                if (i + q * kRowF4 < hi4) count_float4(v[q], rm, cs, t5, t7, acc);
+                if (r + q < first_kept && i + q * kRowF4 < hi4) count_float4(v[q], rm, cs, t5, t7, acc);
             }
+        }
+        for (r = first_kept; r < nrows; ++r) {
+            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
+            if (neg5 || neg7) rm = always;
+            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
+                count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], rm, cs, t5, t7, acc);
         }
         if (owns_tail) {
             const float a = fabsf(tail_u);
@@ -338,6 +356,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         const unsigned int thr16 = __float_as_uint(fmaxf(thr, 0.0f)) >> 16;
         unsigned long long run = sh.base;
         const int trows = nrows < table_rows ? nrows : table_rows;  // rows covered by the table
+        const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
         if (mine != 0u) {
             // step 1: every warp counts the survivors of its qualifying segments; the table
             // entry of a segment is replaced by that count (0 where it cannot qualify).
@@ -378,7 +397,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     if (q < n) {
                         const int r = sh.qrow[w][q];
                         const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                        if (i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                        if (i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
                     }
                 }
 #pragma unroll
@@ -439,7 +458,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     if (q < n) {
                         const int r = sh.qrow[w][q];
                         const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                        if (i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                        if (i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
                     }
                 }
 #pragma unroll
@@ -503,7 +522,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     // warp-uniform: skip the segment when its maximum cannot pass
                     const bool look = r < nrows &&
                                       (all_pass || r >= table_rows || table[r * kFusedWarps + w] > thr16);
-                    if (look && i < hi4) v[q] = (r < cache_rows) ? cache[(size_t)r * kRowF4 + tid] : __ldcg(e4 + i);
+                    if (look && i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
                 }
 #pragma unroll
                 for (int q = 0; q < kGroupRows; ++q) {
@@ -628,6 +647,30 @@ static FusedPlan* fused_plan(int dev, int sm_count) {
     return &p;
 }
 
+// Launch geometry for a vector of d elements on a grid of at most `grid` CTAs.
+struct FusedGeometry {
+    int64_t G;       // CTAs (none without rows)
+    int rpc;         // rows per CTA
+    int u_slots;     // row slots of shared memory that end up holding u
+    int table_rows;  // rows with an entry in the maximum table
+};
+static FusedGeometry fused_geometry(int64_t d, int grid) {
+    FusedGeometry q;
+    const int64_t n4 = d >> 2;
+    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;  // rows in the whole vector
+    int64_t rows_per_cta = (n_rows + grid - 1) / grid;
+    if (rows_per_cta < 1) rows_per_cta = 1;
+    q.G = (n_rows + rows_per_cta - 1) / rows_per_cta;
+    if (q.G < 1) q.G = 1;
+    q.rpc = (int)rows_per_cta;
+    // shared memory: the g ring and the maximum table claim their share, the rest holds u
+    q.table_rows = q.rpc < kTableMaxRows ? q.rpc : kTableMaxRows;
+    const int table_bytes = (q.table_rows * kTableRowBytes + 15) / 16 * 16;
+    q.u_slots = (kFusedSmemBytes - kStages * kRowBytes - table_bytes) / kRowBytes;
+    if (q.u_slots > q.rpc) q.u_slots = q.rpc;
+    return q;
+}
+
 // Returns GK_OK when the fused kernel was enqueued, 1 when it cannot be used on
 // this device or for this call (the caller then takes the three-kernel path),
 // or an error.
@@ -637,19 +680,9 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
     GK_CUDA_TRY(cudaGetDevice(&dev));
     FusedPlan* p = fused_plan(dev, ws->sm_count);
     if (!p || !p->usable || k >= d) return 1;
-    const int64_t n4 = d >> 2;
-    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;  // rows in the whole vector
-    int64_t G = p->grid;
-    int64_t rows_per_cta = (n_rows + G - 1) / G;
-    if (rows_per_cta < 1) rows_per_cta = 1;
-    G = (n_rows + rows_per_cta - 1) / rows_per_cta;  // no CTA without rows
-    if (G < 1) G = 1;
-    int rpc = (int)rows_per_cta;
-    // shared memory: the maximum table first claims its share, the rest caches rows
-    int table_rows = rpc < kTableMaxRows ? rpc : kTableMaxRows;
-    const int table_bytes = (table_rows * kTableRowBytes + 15) / 16 * 16;
-    int cache_rows = (kFusedSmemBytes - table_bytes) / kRowBytes;
-    if (cache_rows > rpc) cache_rows = rpc;
+    FusedGeometry geo = fused_geometry(d, p->grid);
+    int64_t G = geo.G;
+    int rpc = geo.rpc, u_slots = geo.u_slots, table_rows = geo.table_rows;
     const double pq = 1.0 - (double)k / (double)d;  // Algorithm 1: p = 1 - k/d
     double z = normal_quantile_upper(1.0 - pq);
     int64_t cap = output_capacity(d);
@@ -657,7 +690,7 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
     double2* partials = ws->partials;
     unsigned int* cta_counts = ws->cta_counts;
     unsigned int* bars = ws->bars;
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&cache_rows,
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
                     (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
                     (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
     stage_mark(ws, st, 0);
@@ -743,26 +776,17 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
     unsigned int* bars =
         reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes);
 
-    const int64_t n4 = d >> 2;
-    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;
-    int64_t G = plan->grid;
-    int64_t rows_per_cta = (n_rows + G - 1) / G;
-    if (rows_per_cta < 1) rows_per_cta = 1;
-    G = (n_rows + rows_per_cta - 1) / rows_per_cta;
-    if (G < 1) G = 1;
+    FusedGeometry geo = fused_geometry(d, plan->grid);
+    int64_t G = geo.G;
     if (G > kFusedGridCap) return GK_ERR_LIMIT;  // more CTAs than the fixed array has slots for
     // The array keeps what the last call left.  The barrier counters must start at zero; the
     // kernel resets them when it ends, but a call that was cut short would not have.
     GK_CUDA_TRY(cudaMemsetAsync(bars, 0, kStaticBarBytes, st));
-    int rpc = (int)rows_per_cta;
-    int table_rows = rpc < kTableMaxRows ? rpc : kTableMaxRows;
-    const int table_bytes = (table_rows * kTableRowBytes + 15) / 16 * 16;
-    int cache_rows = (kFusedSmemBytes - table_bytes) / kRowBytes;
-    if (cache_rows > rpc) cache_rows = rpc;
+    int rpc = geo.rpc, u_slots = geo.u_slots, table_rows = geo.table_rows;
     const double pq = 1.0 - (double)k / (double)d;
     double z = normal_quantile_upper(1.0 - pq);
     int64_t cap = output_capacity(d);
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&cache_rows,
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
                     (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
                     (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
     GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
