@@ -218,6 +218,15 @@ int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out);
 int gk_stage_timing(int enable);
 int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages);
 
+/*
+ * Per-CTA trace of the last fused gk_sparsify call on `stream` (tracing aid).
+ * Synchronises the stream and writes 8 uint64 per CTA to HOST host_out (room for
+ * 512 x 8): %globaltimer in ns at the CTA's start, before and after the first
+ * grid barrier, before and after the second, and at its end (slots 6, 7 unused).
+ * *n_ctas receives the number of CTAs, 0 if the last call did not run that kernel.
+ */
+int gk_last_cta_trace(gk_stream_t stream, uint64_t* host_out, int* n_ctas);
+
 /* Number of kernels the library has launched so far in this process. */
 int64_t gk_launch_count(void);
 

@@ -22,7 +22,7 @@ GK_DEV_BAD_SEGMENTS = 4
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
-    "gk_stage_timing", "gk_last_stage_ms", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
+    "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
 ]
 
 
@@ -88,6 +88,8 @@ def load() -> C.CDLL:
     L.gk_stage_timing.restype = C.c_int
     L.gk_last_stage_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     L.gk_last_stage_ms.restype = C.c_int
+    L.gk_last_cta_trace.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_int)]
+    L.gk_last_cta_trace.restype = C.c_int
     L.gk_launch_count.argtypes = []
     L.gk_launch_count.restype = i64
     L.gk_strerror.argtypes = [C.c_int]
@@ -220,6 +222,14 @@ def gk_last_stage_ms() -> List[float]:
     n = C.c_int(0)
     _check(load().gk_last_stage_ms(_stream(), ms, C.byref(n)))
     return [float(ms[i]) for i in range(n.value)]
+
+
+def gk_last_cta_trace():
+    """Per-CTA timestamps (ns) of the last fused call on the current stream: list of 8-tuples."""
+    buf = (C.c_uint64 * (512 * 8))()
+    n = C.c_int(0)
+    _check(load().gk_last_cta_trace(_stream(), buf, C.byref(n)))
+    return [tuple(int(buf[i * 8 + j]) for j in range(8)) for i in range(n.value)]
 
 
 def gk_launch_count() -> int:

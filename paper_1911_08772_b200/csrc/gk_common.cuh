@@ -74,6 +74,8 @@ struct Workspace {
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
     unsigned int* cta_counts = nullptr;     // fused kernel: kFusedGridCap x kNumCand
     unsigned int* bars = nullptr;           // fused kernel: two barrier counters and an exit counter
+    unsigned long long* cta_trace = nullptr;  // fused kernel: kFusedGridCap x 8 timestamps (tracing aid)
+    int last_grid = 0;                      // CTAs of the last fused launch
     // segmented call
     void* seg_block = nullptr;
     int sm_count = 0;

@@ -44,13 +44,17 @@ constexpr int kFusedThreads = 1024;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kRowF4 = kFusedThreads;                  // float4 per row
 constexpr int kRowBytes = kRowF4 * 16;                 // 16 KB
-constexpr int kFusedSmemBytes = 13 * kRowBytes;        // dynamic shared memory: g ring, u slots, table
-constexpr int kStages = 4;                             // rows of g (and eps) in flight per CTA, plus one
+constexpr int kTableMaxRows = 224;                     // rows beyond this are ordered in groups and always re-read
+constexpr int kTableBytes = kTableMaxRows * kFusedWarps * 2;  // 14 KB: one uint16 per (row, warp)
+constexpr int kSmemRows = 13;                          // 16 KB rows of dynamic shared memory
+constexpr int kFusedSmemBytes = kSmemRows * kRowBytes + kTableBytes;  // ring, u slots, table
+constexpr int kStages = 4;                             // phase A: rows of g and eps in flight, plus one
+constexpr int kRing = 8;                               // ring slots; phase B has kRing - 1 rows in flight
 constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
-constexpr int kTableMaxRows = 384;                     // rows beyond this are ordered in groups and always re-read
 constexpr int kGroupRows = 8;                          // rows ordered by one in-CTA scan
 constexpr int kFusedMaxGrid = kFusedGridCap;
 constexpr int kBarrierPollLimit = 1 << 24;
+constexpr int kTraceSlots = 8;                         // timestamps per CTA in the optional trace
 
 struct FusedShared {
     double2 red[kFusedWarps];
@@ -145,18 +149,18 @@ __device__ __forceinline__ unsigned int mask_above(const float4 v, const float t
 // rows_per_cta: rows of the run of every CTA; u_slots: row slots of shared memory
 // that receive eps and then hold u (the last u_slots rows of the run stay on
 // chip); table_rows: rows that have an entry in the maximum table.
-// Shared memory: [kStages rows of g in flight][u_slots rows][table].
+// Shared memory: [ring of kRing rows][u_slots rows][table].
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
            int rows_per_cta, int u_slots, int table_rows, Ctrl* __restrict__ ctrl,
            double2* __restrict__ partials, unsigned int* __restrict__ cta_counts,
            unsigned int* __restrict__ bars, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
-           int64_t* __restrict__ nnz_out, int64_t cap) {
+           int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
     extern __shared__ float4 smem4[];
     __shared__ FusedShared sh;
-    float4* gring = smem4;                                   // kStages x kRowF4
-    float4* uslot = smem4 + (size_t)kStages * kRowF4;        // u_slots x kRowF4
-    unsigned short* table = reinterpret_cast<unsigned short*>(uslot + (size_t)u_slots * kRowF4);
+    float4* gring = smem4;                                   // kRing x kRowF4 (phase A uses kStages of them)
+    float4* uslot = smem4 + (size_t)kRing * kRowF4;          // u_slots x kRowF4
+    unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)kSmemRows * kRowF4);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int c = blockIdx.x, G = gridDim.x;
     const int64_t n4 = d >> 2;
@@ -175,6 +179,11 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         ctrl->stats.status = GK_DEV_OK;
         ctrl->phase_t[0] = global_timer_ns();
     }
+    // optional per-CTA trace: start, before / after each barrier, end
+    auto stamp = [&](int slot) {
+        if (trace != nullptr && tid == 0) trace[(size_t)c * kTraceSlots + slot] = global_timer_ns();
+    };
+    stamp(0);
 
     // ------------------------------------------------------------------ phase A
     {
@@ -222,10 +231,12 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         }
         const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
         if (tid == 0) partials[c] = part;
+        stamp(1);
         if (!grid_barrier(&bars[0], (unsigned)G, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
+        stamp(2);
         // every CTA forms the same totals: thread t takes partial t, t + T, ...
         double s = 0.0, q = 0.0;
         for (int i = tid; i < G; i += kFusedThreads) {
@@ -260,21 +271,25 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         const unsigned int always = 0x10000u;  // above every 16-bit maximum
         const bool neg5 = cs[5] < 0.f, neg7 = cs[7] < 0.f;
         const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
-        int r = 0;
-        for (; r < first_kept; r += 4) {
-            float4 v[4];
+        // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
+        // in phase A, kRing - 1 rows ahead of the counting
+        auto fetch_u = [&](int r) {
             const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+            if (r < first_kept && i < hi4) cp_async16(gring + (size_t)(r % kRing) * kRowF4 + tid, e4 + i);
+            cp_async_commit();
+        };
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                v[q] = (r + q < first_kept && i + q * kRowF4 < hi4) ? __ldcg(e4 + i + q * kRowF4)
-                                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                unsigned int rm = (r + q < table_rows) ? table[(r + q) * kFusedWarps + w] : always;
-                if (neg5 || neg7) rm = always;
-                if (r + q < first_kept && i + q * kRowF4 < hi4) count_float4(v[q], rm, cs, t5, t7, acc);
-            }
+        for (int r = 0; r < kRing - 1; ++r) fetch_u(r);
+        int r = 0;
+        for (; r < first_kept; ++r) {
+            fetch_u(r + kRing - 1);
+            cp_async_wait<kRing - 1>();
+            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
+            if (neg5 || neg7) rm = always;
+            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
+                count_float4(gring[(size_t)(r % kRing) * kRowF4 + tid], rm, cs, t5, t7, acc);
         }
+        cp_async_wait<0>();
         for (r = first_kept; r < nrows; ++r) {
             unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
             if (neg5 || neg7) rm = always;
@@ -294,11 +309,13 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         __syncthreads();
         if (tid < kNumCand) cta_counts[(size_t)c * kNumCand + tid] = sh.cta_counts[tid];
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
+        stamp(3);
         if (!grid_barrier(&bars[1], (unsigned)G, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
         if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
+        stamp(4);
     }
 
     // ------------------------------------------------------------------ resolve
@@ -601,6 +618,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     }
 
     if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
+    stamp(5);
 
 leave:
     // the CTA that leaves last clears the barrier counters for the next call
@@ -665,10 +683,22 @@ static FusedGeometry fused_geometry(int64_t d, int grid) {
     q.rpc = (int)rows_per_cta;
     // shared memory: the g ring and the maximum table claim their share, the rest holds u
     q.table_rows = q.rpc < kTableMaxRows ? q.rpc : kTableMaxRows;
-    const int table_bytes = (q.table_rows * kTableRowBytes + 15) / 16 * 16;
-    q.u_slots = (kFusedSmemBytes - kStages * kRowBytes - table_bytes) / kRowBytes;
+    q.u_slots = kSmemRows - kRing;
     if (q.u_slots > q.rpc) q.u_slots = q.rpc;
     return q;
+}
+
+// The one place that builds the kernel's argument list (types checked by the compiler).
+static cudaError_t launch_fused(int64_t G, cudaStream_t st, const float* g, float* eps, int64_t d, int64_t k, double z,
+                                int rpc, int u_slots, int table_rows, Ctrl* ctrl, double2* partials,
+                                unsigned int* cta_counts, unsigned int* bars, int32_t* idx_out, float* val_out,
+                                int64_t* nnz_out, int64_t cap, unsigned long long* trace) {
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
+                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
+                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap, (void*)&trace};
+    static_assert(sizeof(args) / sizeof(args[0]) == 17, "k_gk_fused takes 17 arguments");
+    return cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
+                                       (size_t)kFusedSmemBytes, st);
 }
 
 // Returns GK_OK when the fused kernel was enqueued, 1 when it cannot be used on
@@ -690,12 +720,11 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
     double2* partials = ws->partials;
     unsigned int* cta_counts = ws->cta_counts;
     unsigned int* bars = ws->bars;
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
-                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
-                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
+    unsigned long long* trace = ws->cta_trace;
+    ws->last_grid = (int)G;
     stage_mark(ws, st, 0);
-    GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
-                                            (size_t)kFusedSmemBytes, st));
+    GK_CUDA_TRY(launch_fused(G, st, g, eps, d, k, z, rpc, u_slots, table_rows, ctrl, partials, cta_counts, bars,
+                             idx_out, val_out, nnz_out, cap, trace));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_fused = true;
@@ -786,11 +815,9 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
     const double pq = 1.0 - (double)k / (double)d;
     double z = normal_quantile_upper(1.0 - pq);
     int64_t cap = output_capacity(d);
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
-                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
-                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap};
-    GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
-                                            (size_t)kFusedSmemBytes, st));
+    unsigned long long* trace = nullptr;  // no trace array in the fixed scratch
+    GK_CUDA_TRY(launch_fused(G, st, g, eps, d, k, z, rpc, u_slots, table_rows, ctrl, partials, cta_counts, bars,
+                             idx_out, val_out, nnz_out, cap, trace));
     note_launch();
     return GK_OK;
 }

@@ -49,7 +49,7 @@ int64_t output_capacity(int64_t d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t ctrl, partials, hist, cta_counts, bars, tile_status, seg, total;
+    size_t ctrl, partials, hist, cta_counts, bars, cta_trace, tile_status, seg, total;
 };
 
 static Layout layout_for(int64_t d, int32_t S) {
@@ -60,6 +60,7 @@ static Layout layout_for(int64_t d, int32_t S) {
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
     L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
     L.bars = at;        at = align_up(at + sizeof(unsigned int) * 4, 256);
+    L.cta_trace = at;   at = align_up(at + sizeof(unsigned long long) * kFusedGridCap * 8, 256);
     L.tile_status = at; at = align_up(at + sizeof(unsigned long long) * (size_t)num_compact_tiles(d), 256);
     L.seg = at;         at = align_up(at + segmented_scratch_bytes(d, S), 256);
     L.total = at;
@@ -96,6 +97,7 @@ int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out
         ws.hist = reinterpret_cast<unsigned int*>(b + L.hist);
         ws.cta_counts = reinterpret_cast<unsigned int*>(b + L.cta_counts);
         ws.bars = reinterpret_cast<unsigned int*>(b + L.bars);
+        ws.cta_trace = reinterpret_cast<unsigned long long*>(b + L.cta_trace);
         ws.tile_status = reinterpret_cast<unsigned long long*>(b + L.tile_status);
         ws.seg_block = b + L.seg;
         GK_CUDA_TRY(cudaDeviceGetAttribute(&ws.sm_count, cudaDevAttrMultiProcessorCount, dev));
@@ -195,6 +197,18 @@ extern "C" int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages
         for (int i = 0; i < 6; ++i) ms_out[1 + i] = (float)((double)(t[i + 1] - t[i]) * 1e-6);
         *n_stages = 7;
     }
+    return GK_OK;
+}
+
+extern "C" int gk_last_cta_trace(gk_stream_t stream, uint64_t* host_out, int* n_ctas) {
+    if (!host_out || !n_ctas) return GK_ERR_NULL;
+    Workspace* ws = find_workspace((cudaStream_t)stream);
+    if (!ws) return GK_ERR_NULL;
+    GK_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    *n_ctas = ws->last_fused ? ws->last_grid : 0;
+    if (*n_ctas > 0)
+        GK_CUDA_TRY(cudaMemcpy(host_out, ws->cta_trace, sizeof(uint64_t) * 8 * (size_t)*n_ctas,
+                               cudaMemcpyDeviceToHost));
     return GK_OK;
 }
 
