@@ -85,6 +85,14 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// 32-byte store that asks L2 to keep the line longer than ordinary traffic (the eviction
+// priority is only available on 256-bit accesses).  p must be 32-byte aligned.
+__device__ __forceinline__ void st_keep32(float4* p, const float4 a, const float4 b) {
+    asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(a.x), "f"(a.y),
+                 "f"(a.z), "f"(a.w), "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
+                 : "memory");
+}
+
 // Arrive at a barrier counter and wait until all G CTAs have arrived.
 // Returns false when the bounded wait ran out.
 __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int G, int* ok_flag) {
@@ -125,15 +133,21 @@ __device__ __forceinline__ void count_tier(const float a0, const float a1, const
 }
 
 // rm: the segment's largest magnitude (top 16 bits, rounded up).  A candidate whose top 16
-// bits (rounded down) are not below rm cannot be exceeded by any element of the segment.
+// bits (rounded down) are not below rm cannot be exceeded by any element of the segment, nor
+// can any larger candidate: candidates 0..1, 2..4, 5..6 and 7..9 (in ascending order) are
+// evaluated only as far as the segment's maximum reaches.
+struct Tiers { unsigned int t0, t2, t5, t7; };
 __device__ __forceinline__ void count_float4(const float4 v, const unsigned int rm, const float (&cs)[kNumCand],
-                                             const unsigned int t5, const unsigned int t7,
-                                             float (&acc)[kNumCand]) {
+                                             const Tiers& tier, float (&acc)[kNumCand]) {
+    if (rm <= tier.t0) return;  // warp-uniform, as are the tests below
     const float a0 = fabsf(v.x), a1 = fabsf(v.y), a2 = fabsf(v.z), a3 = fabsf(v.w);
-    count_tier<0, 5>(a0, a1, a2, a3, cs, acc);
-    if (rm > t5) {  // warp-uniform
-        count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
-        if (rm > t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
+    count_tier<0, 2>(a0, a1, a2, a3, cs, acc);
+    if (rm > tier.t2) {
+        count_tier<2, 5>(a0, a1, a2, a3, cs, acc);
+        if (rm > tier.t5) {
+            count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
+            if (rm > tier.t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
+        }
     }
 }
 
@@ -175,6 +189,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     const float4* g4 = reinterpret_cast<const float4*>(g);
     float4* e4 = reinterpret_cast<float4*>(eps);
     float tail_u = 0.f;
+    const bool wide_ok = ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
     if (c == 0 && tid == 0) {
         ctrl->stats.status = GK_DEV_OK;
         ctrl->phase_t[0] = global_timer_ns();
@@ -211,12 +226,25 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
                 const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *us;
                 u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
-                e4[i] = u0;
                 *us = u0;
                 const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
                              x3 = (double)u0.w - pv;
                 s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
                 s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
+            }
+            // u goes out in 32-byte stores by the even lanes (own float4 and the right neighbour's),
+            // marked to stay in L2: the next two phases read most of u again
+            {
+                float4 nb;
+                nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
+                nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
+                const bool pair = wide_ok && (i + 1 < hi4);  // this lane and its right neighbour are in range
+                if ((lane & 1) == 0) {
+                    if (pair) st_keep32(e4 + i, u0, nb);
+                    else if (one) e4[i] = u0;
+                } else if (one && !wide_ok) {
+                    e4[i] = u0;
+                }
             }
             // largest magnitude of each (row, warp) segment, top 16 bits rounded up
             const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
@@ -265,36 +293,46 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         float cs[kNumCand], acc[kNumCand];
 #pragma unroll
         for (int j = 0; j < kNumCand; ++j) { cs[j] = sh.cand32[sh.order[j]]; acc[j] = 0.f; }
-        // tiers: candidates 5..6 and 7..9 are evaluated only for segments whose maximum can pass
-        const unsigned int t5 = cs[5] < 0.f ? 0u : (__float_as_uint(cs[5]) >> 16);
-        const unsigned int t7 = cs[7] < 0.f ? 0u : (__float_as_uint(cs[7]) >> 16);
+        // tier limits: top 16 bits of the tier's lowest candidate, rounded down; a negative
+        // candidate is exceeded by everything, and candidates ascend, so testing the lowest suffices
+        Tiers tier;
+        tier.t0 = __float_as_uint(fmaxf(cs[0], 0.f)) >> 16;
+        tier.t2 = __float_as_uint(fmaxf(cs[2], 0.f)) >> 16;
+        tier.t5 = __float_as_uint(fmaxf(cs[5], 0.f)) >> 16;
+        tier.t7 = __float_as_uint(fmaxf(cs[7], 0.f)) >> 16;
         const unsigned int always = 0x10000u;  // above every 16-bit maximum
-        const bool neg5 = cs[5] < 0.f, neg7 = cs[7] < 0.f;
+        const bool any_neg = cs[0] < 0.f;
         const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
+        // only the last row of a run can be short: `mine_last` says whether this thread has a part in it
+        const int nfull = (int)((hi4 - lo4) / kRowF4);
+        const bool mine_last = lo4 + (int64_t)nfull * kRowF4 + tid < hi4;
+        const float4* src = e4 + lo4 + tid;
+        const unsigned short* trow = table + w;
         // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
         // in phase A, kRing - 1 rows ahead of the counting
         auto fetch_u = [&](int r) {
-            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-            if (r < first_kept && i < hi4) cp_async16(gring + (size_t)(r % kRing) * kRowF4 + tid, e4 + i);
+            if (r < first_kept && (r < nfull || mine_last))
+                cp_async16(gring + ((r & (kRing - 1)) << 10) + tid, src + ((size_t)r << 10));
             cp_async_commit();
+        };
+        auto row_max = [&](int r) -> unsigned int {
+            return (any_neg || r >= table_rows) ? always : (unsigned int)trow[r * kFusedWarps];
         };
 #pragma unroll
         for (int r = 0; r < kRing - 1; ++r) fetch_u(r);
+        static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
         int r = 0;
+#pragma unroll 2
         for (; r < first_kept; ++r) {
             fetch_u(r + kRing - 1);
             cp_async_wait<kRing - 1>();
-            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
-            if (neg5 || neg7) rm = always;
-            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
-                count_float4(gring[(size_t)(r % kRing) * kRowF4 + tid], rm, cs, t5, t7, acc);
+            if (r < nfull || mine_last)
+                count_float4(gring[((r & (kRing - 1)) << 10) + tid], row_max(r), cs, tier, acc);
         }
         cp_async_wait<0>();
         for (r = first_kept; r < nrows; ++r) {
-            unsigned int rm = (r < table_rows) ? table[r * kFusedWarps + w] : always;
-            if (neg5 || neg7) rm = always;
-            if (lo4 + (int64_t)r * kRowF4 + tid < hi4)
-                count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], rm, cs, t5, t7, acc);
+            if (r < nfull || mine_last)
+                count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], row_max(r), cs, tier, acc);
         }
         if (owns_tail) {
             const float a = fabsf(tail_u);
