@@ -70,48 +70,104 @@ __device__ __forceinline__ unsigned int tile_scan(const unsigned int (&c)[kCompa
     return sm.total;
 }
 
-// Look-back by one full warp.  `aggregate` is this tile's payload (< 2^62; the
-// exact Top_k path packs two 31-bit counts, whose sums never carry into each
-// other because d < 2^31).  Returns the sum of the payloads of all earlier
-// tiles and publishes this tile's inclusive prefix.
-__device__ __forceinline__ unsigned long long lookback_warp(unsigned long long* status, int tile,
-                                                            unsigned long long aggregate,
-                                                            int* dev_status) {
-    const int lane = threadIdx.x & 31;
+// Look-back by the whole CTA: every thread inspects one predecessor, so one round trip to
+// memory covers kCompactThreads tiles (with a few hundred tiles in flight at once, a
+// warp-wide window would need many round trips to reach a tile that already knows its
+// prefix).  `aggregate` is this tile's payload (< 2^62; the exact Top_k path packs two
+// 31-bit counts, whose sums never carry into each other because d < 2^31).  Called by all
+// threads; returns to all of them the sum of the payloads of all earlier tiles, and
+// publishes this tile's inclusive prefix.
+struct LookbackSmem {
+    unsigned long long sum_all[kCompactThreads / 32];
+    unsigned long long sum_upto[kCompactThreads / 32];
+    int first[kCompactThreads / 32];  // lane of the nearest prefix holder in the warp, 32 if none
+    int gave_up;
+    unsigned long long result;
+};
+
+__device__ __forceinline__ unsigned long long lookback_block(unsigned long long* status, int tile,
+                                                             unsigned long long aggregate, int* dev_status,
+                                                             LookbackSmem& sm) {
+    constexpr int NW = kCompactThreads / 32;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     if (tile == 0) {
-        if (lane == 0) st_status(&status[0], (kFlagPrefix << kFlagShift) | aggregate);
+        if (tid == 0) st_status(&status[0], (kFlagPrefix << kFlagShift) | aggregate);
         return 0ull;
     }
-    if (lane == 0) st_status(&status[tile], (kFlagAggregate << kFlagShift) | aggregate);
+    if (tid == 0) {
+        st_status(&status[tile], (kFlagAggregate << kFlagShift) | aggregate);
+        sm.gave_up = 0;
+    }
+    __syncthreads();
     unsigned long long excl = 0ull;
     int pos = tile - 1;
-    bool gave_up = false;
     while (true) {
-        const int mine = pos - lane;
+        const int mine = pos - tid;
         // before tile 0 sits a virtual inclusive prefix of zero
         unsigned long long wd = (mine >= 0) ? ld_status(&status[mine]) : (kFlagPrefix << kFlagShift);
         int polls = 0;
-        while (__any_sync(0xffffffffu, (wd >> kFlagShift) == 0ull)) {
-            if (++polls > kLookbackPollLimit) { gave_up = true; break; }
+        while ((wd >> kFlagShift) == 0ull) {  // bounded wait for this predecessor's word
+            if (++polls > kLookbackPollLimit) { sm.gave_up = 1; break; }
             __nanosleep(20);
-            if ((wd >> kFlagShift) == 0ull) wd = ld_status(&status[mine]);
+            wd = ld_status(&status[mine]);
         }
-        if (gave_up) break;
         const unsigned int pm = __ballot_sync(0xffffffffu, (wd >> kFlagShift) == kFlagPrefix);
-        const int stop = pm ? (__ffs(pm) - 1) : 31;  // nearest predecessor holding a prefix
-        unsigned long long v = (lane <= stop) ? (wd & kPayloadMask) : 0ull;
+        const int fl = pm ? (__ffs(pm) - 1) : 32;
+        unsigned long long all = wd & kPayloadMask;
+        unsigned long long upto = (lane <= fl) ? all : 0ull;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        excl += v;
-        if (pm) break;
-        pos -= 32;
+        for (int o = 16; o > 0; o >>= 1) {
+            all += __shfl_xor_sync(0xffffffffu, all, o);
+            upto += __shfl_xor_sync(0xffffffffu, upto, o);
+        }
+        if (lane == 0) { sm.sum_all[w] = all; sm.sum_upto[w] = upto; sm.first[w] = fl; }
+        __syncthreads();
+        // warps are in order of distance: the first warp that holds a prefix ends the walk
+        unsigned long long total = 0ull;
+        bool found = false;
+#pragma unroll
+        for (int q = 0; q < NW; ++q) {
+            if (!found) {
+                if (sm.first[q] < 32) { total += sm.sum_upto[q]; found = true; }
+                else total += sm.sum_all[q];
+            }
+        }
+        const bool stop = found || sm.gave_up;
+        excl += total;
+        __syncthreads();  // the arrays are rewritten by the next window
+        if (stop) break;
+        pos -= kCompactThreads;
     }
-    if (gave_up) {
-        if (lane == 0) atomicOr(dev_status, GK_DEV_TIMEOUT);
+    if (sm.gave_up) {
+        if (tid == 0) atomicOr(dev_status, GK_DEV_TIMEOUT);
         excl = 0ull;
     }
-    if (lane == 0) st_status(&status[tile], (kFlagPrefix << kFlagShift) | (excl + aggregate));
+    if (tid == 0) st_status(&status[tile], (kFlagPrefix << kFlagShift) | (excl + aggregate));
     return excl;
+}
+
+// Host side: launch a compaction kernel whose last parameter is the `persistent` flag.
+// Where the device supports it the kernel is launched cooperatively with as many CTAs as are
+// resident at once (persistent = 1: static tile assignment, no ticket); otherwise one CTA per
+// tile with ticketed tiles.  The arguments must have exactly the kernel's parameter types.
+template <class Kernel, class... Args>
+inline cudaError_t launch_compaction(Kernel kernel, int n_tiles, int sm_count, cudaStream_t st, Args... a) {
+    int dev = 0, coop = 0, occ = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    int persistent = 0;
+    int grid = n_tiles;
+    if (coop && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kCompactThreads, 0) == cudaSuccess &&
+        occ > 0) {
+        persistent = 1;
+        grid = occ * sm_count < n_tiles ? occ * sm_count : n_tiles;
+    } else {
+        cudaGetLastError();
+    }
+    void* args[] = {(void*)&a..., (void*)&persistent};
+    if (persistent)
+        return cudaLaunchCooperativeKernel((const void*)kernel, dim3((unsigned)grid), dim3(kCompactThreads), args, 0, st);
+    return cudaLaunchKernel((const void*)kernel, dim3((unsigned)grid), dim3(kCompactThreads), args, 0, st);
 }
 
 }  // namespace gk

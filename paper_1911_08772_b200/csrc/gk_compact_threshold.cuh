@@ -27,15 +27,26 @@ k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
                     unsigned long long* __restrict__ tile_status, int n_tiles,
                     int32_t* __restrict__ idx_out, float* __restrict__ val_out,
                     int64_t* __restrict__ nnz_out, int64_t cap,
-                    const int64_t* __restrict__ seg_off, int S, const float* __restrict__ seg_thr) {
+                    const int64_t* __restrict__ seg_off, int S, const float* __restrict__ seg_thr,
+                    int persistent) {
     __shared__ TileScanSmem scan;
     __shared__ int s_tile;
-    __shared__ unsigned long long s_prefix;
+    __shared__ LookbackSmem lb;
     __shared__ unsigned int s_tailcnt;
     const int tid = threadIdx.x;
-    if (tid == 0) {
-        s_tile = (int)atomicAdd(&ctrl->tile_ticket, 1u);
-        s_tailcnt = 0u;
+    // persistent: launched cooperatively with all CTAs resident, CTA b takes tiles b, b + grid, ...
+    // (every earlier tile belongs to a resident CTA, so the look-back always makes progress);
+    // otherwise one tile per CTA, handed out by an atomic ticket in the order the CTAs start.
+    for (int pass = 0;; ++pass) {
+    if (persistent) {
+        if ((int64_t)blockIdx.x + (int64_t)pass * gridDim.x >= n_tiles) break;
+        if (tid == 0) { s_tile = (int)(blockIdx.x + pass * gridDim.x); s_tailcnt = 0u; }
+    } else {
+        if (pass > 0) break;
+        if (tid == 0) {
+            s_tile = (int)atomicAdd(&ctrl->tile_ticket, 1u);
+            s_tailcnt = 0u;
+        }
     }
     __syncthreads();
     const int tile = s_tile;
@@ -106,13 +117,8 @@ k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
     const unsigned int total = tile_scan(c, off, scan);  // synchronises the CTA
     const unsigned int tile_total = total + s_tailcnt;
 
-    if (tid < 32) {
-        const unsigned long long excl =
-            lookback_warp(tile_status, tile, (unsigned long long)tile_total, &ctrl->stats.status);
-        if (tid == 0) s_prefix = excl;
-    }
-    __syncthreads();
-    const unsigned long long prefix = s_prefix;
+    const unsigned long long prefix =
+        lookback_block(tile_status, tile, (unsigned long long)tile_total, &ctrl->stats.status, lb);
 
     if (mask) {
 #pragma unroll
@@ -156,6 +162,8 @@ k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
         ctrl->stats.emitted = written;
         if (all > cap) atomicOr(&ctrl->stats.status, GK_DEV_TRUNCATED);
         ctrl->tile_ticket = 0u;
+    }
+    __syncthreads();  // shared arrays are reused by the next tile
     }
 }
 

@@ -299,9 +299,9 @@ extern "C" int gk_sparsify_segmented(const float* g, float* eps, int64_t d, cons
                                                            ws->tile_status, n_tiles);
     k_seg_count_candidates<<<(int)G, kSegThreads, 0, st>>>(eps, d, r4, seg_offsets, seg_k, S, ws->ctrl, v,
                                                            seg_nnz_out);
-    k_compact_threshold<true><<<n_tiles, kCompactThreads, 0, st>>>(eps, d, ws->ctrl, ws->tile_status, n_tiles,
-                                                                  idx_out, val_out, nnz_out,
-                                                                  output_capacity(d), seg_offsets, S, v.thr_sel);
+    GK_CUDA_TRY(launch_compaction(k_compact_threshold<true>, n_tiles, ws->sm_count, st, eps, d, ws->ctrl,
+                                  ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
+                                  seg_offsets, (int)S, (const float*)v.thr_sel));
     note_launch(3);
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;

@@ -220,9 +220,9 @@ int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d
         note_launch();
     }
     stage_mark(ws, st, 2);
-    k_compact_threshold<false><<<n_tiles, kCompactThreads, 0, st>>>(
-        eps, d, ws->ctrl, ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d), nullptr, 0,
-        nullptr);
+    GK_CUDA_TRY(launch_compaction(k_compact_threshold<false>, n_tiles, ws->sm_count, st, eps, d, ws->ctrl,
+                                  ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
+                                  (const int64_t*)nullptr, 0, (const float*)nullptr));
     note_launch();
     stage_mark(ws, st, 3);
     ws->last_fused = false;

@@ -134,19 +134,27 @@ template <bool CLEAR>
 __global__ void __launch_bounds__(kCompactThreads)
 k_compact_topk(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
                unsigned long long* __restrict__ tile_status, int n_tiles,
-               int32_t* __restrict__ idx_out, float* __restrict__ val_out) {
+               int32_t* __restrict__ idx_out, float* __restrict__ val_out, int persistent) {
     __shared__ TileScanSmem scan;
     __shared__ int s_tile;
-    __shared__ unsigned long long s_prefix;
+    __shared__ LookbackSmem lb;
     __shared__ unsigned int s_tail_gt, s_tail_eq;
     const int tid = threadIdx.x;
-    if (tid == 0) {
-        s_tile = (int)atomicAdd(&ctrl->tile_ticket, 1u);
-        s_tail_gt = 0u;
-        s_tail_eq = 0u;
-    }
     const unsigned int T = ctrl->key_threshold;
     const unsigned long long need_eq = ctrl->need_eq;
+    // persistent: cooperative launch, CTA b takes tiles b, b + grid, ...; else one ticketed tile
+    for (int pass = 0;; ++pass) {
+    if (persistent) {
+        if ((int64_t)blockIdx.x + (int64_t)pass * gridDim.x >= n_tiles) break;
+        if (tid == 0) { s_tile = (int)(blockIdx.x + pass * gridDim.x); s_tail_gt = 0u; s_tail_eq = 0u; }
+    } else {
+        if (pass > 0) break;
+        if (tid == 0) {
+            s_tile = (int)atomicAdd(&ctrl->tile_ticket, 1u);
+            s_tail_gt = 0u;
+            s_tail_eq = 0u;
+        }
+    }
     __syncthreads();
     const int tile = s_tile;
     const int64_t n4 = d >> 2;
@@ -192,13 +200,9 @@ k_compact_topk(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
     const unsigned int tot_eq = tile_scan(ce, oe, scan);
     const unsigned long long agg =
         (unsigned long long)(tot_gt + s_tail_gt) | ((unsigned long long)(tot_eq + s_tail_eq) << 31);
-    if (tid < 32) {
-        const unsigned long long excl = lookback_warp(tile_status, tile, agg, &ctrl->stats.status);
-        if (tid == 0) s_prefix = excl;
-    }
-    __syncthreads();
-    const unsigned long long pre_gt = s_prefix & 0x7fffffffull;
-    const unsigned long long pre_eq = s_prefix >> 31;
+    const unsigned long long excl = lookback_block(tile_status, tile, agg, &ctrl->stats.status, lb);
+    const unsigned long long pre_gt = excl & 0x7fffffffull;
+    const unsigned long long pre_eq = excl >> 31;
 
     if (mgt | meq) {
 #pragma unroll
@@ -236,6 +240,8 @@ k_compact_topk(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
         }
     }
     if (tile == n_tiles - 1 && tid == 0) ctrl->tile_ticket = 0u;
+    __syncthreads();  // shared arrays are reused by the next tile
+    }
 }
 
 // u = g + eps stored over eps (Eq. 2), no statistics.
@@ -278,8 +284,8 @@ static int enqueue_topk(Workspace* ws, float* u, int64_t d, int64_t k, int32_t* 
     stage_mark(ws, st, ev0 + 2);
     k_radix_histogram<2><<<grid, kHistThreads, 0, st>>>(u, d, k, ws->ctrl, ws->hist, ws->tile_status, n_tiles);
     stage_mark(ws, st, ev0 + 3);
-    k_compact_topk<CLEAR><<<n_tiles, kCompactThreads, 0, st>>>(u, d, ws->ctrl, ws->tile_status, n_tiles,
-                                                             idx_out, val_out);
+    GK_CUDA_TRY(launch_compaction(k_compact_topk<CLEAR>, n_tiles, ws->sm_count, st, u, d, ws->ctrl, ws->tile_status,
+                                  n_tiles, idx_out, val_out));
     stage_mark(ws, st, ev0 + 4);
     note_launch(4);
     GK_CUDA_TRY(cudaGetLastError());
