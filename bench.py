@@ -2,7 +2,7 @@
 """Benchmark of the error-compensated Gaussian_k sparsifier on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload NAME] [--path 0|1] [--loop-only]
+                    [--workload NAME] [--path 0|1] [--loop-only] [--sweep]
 
 One "step" is one whole pass of the hot path -- gk_sparsify(g, eps, d, k, ...) -- over one
 synthetic gradient vector with the residual eps carried from step to step.  The default
@@ -400,6 +400,82 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Every workload family at 1 GPU: Gaussian_k (fused kernel), the segmented call where the
+    workload has segments, and exact Top_k, each timed with CUDA events over a few EC steps
+    with fresh gradients; one JSON object per line on stdout."""
+    import torch
+
+    from paper_1911_08772_b200 import binding as gk
+    from paper_1911_08772_b200 import build as lib_build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    lib_build.build()
+    gk.load()
+    peak, peak_src = measured_peaks()
+    points = [(wl.resnet20_normal(), ["1e-3"]), (wl.vgg16_laplace_mixture(), ["1e-3"]),
+              (wl.resnet50_segmented(), ["1e-3", "1e-2"]), (wl.lstm_student_t(), ["1e-3", "5e-3"])]
+    for lg in (20, 22, 24, 26, 28):
+        for dist in ("normal", "laplace"):
+            points.append((wl.sweep_point(1 << lg, dist), ["1e-4", "1e-3", "1e-2"]))
+    n_grad = 4
+    for w, rhos in points:
+        d = w.d
+        gs = [torch.from_numpy(w.grad(j, None)).to(dev) for j in range(n_grad)]
+        eps = torch.zeros(d, dtype=torch.float32, device=dev)
+        idx = torch.empty(d, dtype=torch.int32, device=dev)
+        val = torch.empty(d, dtype=torch.float32, device=dev)
+        nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+        gk.gk_reserve(d, 161)
+        reps = 40 if d <= (1 << 26) else 12
+        for rho in rhos:
+            k = w.k(rho)
+
+            def timed(fn):
+                # EC episodes of n_grad steps from eps = 0, as many as fit `reps` steps
+                for t in range(3):
+                    fn(t)
+                ms = 0.0
+                for e in range(max(1, reps // n_grad)):
+                    eps.zero_()
+                    ms += time_region(torch, fn, n_grad)
+                return ms / (max(1, reps // n_grad) * n_grad)
+
+            ms_gk = timed(lambda t: gk.gk_sparsify(gs[t % n_grad], eps, k, idx, val, nnz))
+            n_gk = int(nnz.item())
+            st = gk.gk_last_stats()
+            rec = {"workload": w.name, "d": d, "rho": rho, "k": k, "gaussiank_ms": ms_gk,
+                   "gaussiank_gbs": algorithmic_bytes(d, n_gk) / ms_gk / 1e6,
+                   "gaussiank_elements_per_s": d / (ms_gk * 1e-3),
+                   "frac_of_measured_hbm": algorithmic_bytes(d, n_gk) / ms_gk / 1e6 / peak,
+                   "frac_of_nominal_8TBs": algorithmic_bytes(d, n_gk) / ms_gk / 1e6 / 8000.0,
+                   "nnz_last": n_gk, "rounds_last": st.rounds}
+            if w.partition is not None:
+                part = w.partition
+                off = torch.from_numpy(part.offsets).to(dev)
+                sk = torch.from_numpy(part.seg_k(*wl.RHO[rho])).to(dev)
+                snn = torch.zeros(part.S, dtype=torch.int64, device=dev)
+                ms_seg = timed(lambda t: gk.gk_sparsify_segmented(gs[t % n_grad], eps, off, sk, idx, val, snn, nnz))
+                rec["segmented_ms"] = ms_seg
+                rec["segmented_gbs"] = algorithmic_bytes(d, int(nnz.item())) / ms_seg / 1e6
+            u = gs[0]
+            tk_i = torch.empty(k, dtype=torch.int32, device=dev)
+            tk_v = torch.empty(k, dtype=torch.float32, device=dev)
+            for _ in range(3):
+                gk.topk_exact(u, k, tk_i, tk_v)
+            ms_tk = time_region(torch, lambda t: gk.topk_exact(u, k, tk_i, tk_v), 10) / 10
+            ms_tks = timed(lambda t: gk.topk_sparsify(gs[t % n_grad], eps, k, tk_i, tk_v, nnz))
+            rec.update({"topk_exact_ms": ms_tk, "topk_sparsify_ms": ms_tks,
+                        "speedup_vs_topk_sparsify": ms_tks / ms_gk,
+                        "topk_exact_gbs_12B_per_elem": 12.0 * d / ms_tk / 1e6})
+            print(json.dumps(rec), flush=True)
+        del gs, eps, idx, val
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -413,8 +489,12 @@ def main():
                     help="number of gradient buffers kept on the device (default 20; small for captures)")
     ap.add_argument("--loop-only", action="store_true",
                     help="run only warm-up and the timed loop (for profiler captures)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every workload family (Gaussian_k, segmented, exact Top_k) and print one line each")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
