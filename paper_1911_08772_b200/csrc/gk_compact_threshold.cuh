@@ -9,11 +9,26 @@
 namespace gk {
 
 // Segment that holds element i: the s in [0, S) with off[s] <= i < off[s + 1].
+// Called by all 32 lanes of a warp with the same arguments: a 32-ary search, so that a table
+// of a few hundred segments costs two rounds of global loads instead of eight.
 __device__ __forceinline__ int find_segment(const int64_t* __restrict__ off, int S, int64_t i) {
-    int lo = 0, hi = S - 1;  // first s with off[s + 1] > i
+    const int lane = threadIdx.x & 31;
+    int lo = 0, hi = S - 1;  // the answer is the first s in [lo, hi] with off[s + 1] > i
     while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (off[mid + 1] > i) hi = mid; else lo = mid + 1;
+        const int n = hi - lo + 1;
+        const int step = (n + 31) / 32;
+        // lane l asks about the last segment of its group: s_l = lo + (l + 1) * step - 1
+        int sl = lo + (lane + 1) * step - 1;
+        if (sl > hi) sl = hi;
+        const bool above = off[sl + 1] > i;
+        const unsigned int m = __ballot_sync(0xffffffffu, above);
+        if (m == 0u) { lo = hi; break; }  // malformed table: settle on the last segment
+        const int g = __ffs(m) - 1;       // first group whose last segment ends above i
+        int nhi = lo + (g + 1) * step - 1;
+        if (nhi > hi) nhi = hi;
+        lo = lo + g * step;
+        hi = nhi;
+        if (step == 1) { lo = hi; break; }
     }
     return lo;
 }

@@ -37,6 +37,7 @@
 
 #include "gk_alg1.cuh"
 #include "gk_common.cuh"
+#include "gk_count.cuh"
 
 namespace gk {
 
@@ -113,46 +114,6 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
     }
     __syncthreads();
     return *ok_flag != 0;
-}
-
-// 1.0f when a > c, else 0.0f: one compare instruction with a float result.
-__device__ __forceinline__ float gt_as_float(float a, float c) {
-    float r;
-    asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(c));
-    return r;
-}
-
-// Candidates LO..HI-1 (in ascending order of value) against the four magnitudes of one
-// float4.  The counters are floats: exact up to 2^24 per thread, far above a thread's share.
-template <int LO, int HI>
-__device__ __forceinline__ void count_tier(const float a0, const float a1, const float a2, const float a3,
-                                           const float (&cs)[kNumCand], float (&acc)[kNumCand]) {
-#pragma unroll
-    for (int j = LO; j < HI; ++j)
-        acc[j] += (gt_as_float(a0, cs[j]) + gt_as_float(a1, cs[j])) + (gt_as_float(a2, cs[j]) + gt_as_float(a3, cs[j]));
-}
-
-// rm: the segment's largest magnitude (top 16 bits, rounded up).  A candidate whose top 16
-// bits (rounded down) are not below rm cannot be exceeded by any element of the segment, nor
-// can any larger candidate: candidates 0..1, 2..4, 5..6 and 7..9 (in ascending order) are
-// evaluated only as far as the segment's maximum reaches.
-struct Tiers { unsigned int t0, t2, t5, t7; };
-__device__ __forceinline__ void count_float4(const float4 v, const unsigned int rm, const float (&cs)[kNumCand],
-                                             const Tiers& tier, float (&acc)[kNumCand]) {
-    if (rm <= tier.t0) return;  // warp-uniform, as are the tests below
-    const float a0 = fabsf(v.x), a1 = fabsf(v.y), a2 = fabsf(v.z), a3 = fabsf(v.w);
-    count_tier<0, 2>(a0, a1, a2, a3, cs, acc);
-    if (rm > tier.t2) {
-        count_tier<2, 5>(a0, a1, a2, a3, cs, acc);
-        if (rm > tier.t5) {
-            count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
-            if (rm > tier.t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
-        }
-    }
-}
-
-__device__ __forceinline__ unsigned int max_mag_bits(const float4 u) {
-    return __float_as_uint(fmaxf(fmaxf(fabsf(u.x), fabsf(u.y)), fmaxf(fabsf(u.z), fabsf(u.w))));
 }
 
 __device__ __forceinline__ unsigned int mask_above(const float4 v, const float thr) {

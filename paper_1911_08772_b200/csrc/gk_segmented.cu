@@ -15,11 +15,13 @@
 #include "gk_common.cuh"
 #include "gk_compact.cuh"
 #include "gk_compact_threshold.cuh"
+#include "gk_count.cuh"
 #include "gk_segmented.cuh"
 
 namespace gk {
 
 constexpr int kSegThreads = 512;
+constexpr int kSegWindow = 128;  // segments whose scalars a CTA keeps in shared memory at a time
 
 struct Span {
     int64_t lo, hi;      // elements [lo, hi)
@@ -71,20 +73,51 @@ k_seg_accumulate_stats(const float* __restrict__ g, float* __restrict__ eps, int
     for (int64_t t = (int64_t)c * kSegThreads + tid; t < n_tiles; t += (int64_t)G * kSegThreads)
         tile_status[t] = 0ull;
 
+    // the normal quantiles depend only on (k_s, d_s): thread t of CTA c takes segment c + t * G
+    // now, while the other threads stream, so that the finalising CTA only has to read them
+    {
+        const int64_t q = (int64_t)c + (int64_t)tid * G;
+        if (q < S) {
+            const int64_t n = off[q + 1] - off[q];
+            int64_t kk = seg_k[q];
+            if (kk > n) kk = n;
+            double zq = -INFINITY;
+            if (n > 0 && kk >= 1 && kk < n) {
+                const double p = 1.0 - (double)kk / (double)n;  // Algorithm 1: p = 1 - k/d
+                zq = normal_quantile_upper(1.0 - p);
+            }
+            v.zs[q] = zq;
+        }
+    }
     int64_t lo, hi;
     cta_range(c, G, r4, d, &lo, &hi);
     const float4* g4 = reinterpret_cast<const float4*>(g);
     float4* e4 = reinterpret_cast<float4*>(eps);
     int s = (lo < hi) ? find_segment(off, S, lo) : S;
     int64_t cur = lo;
+    // offsets and pivots of the next kSegWindow segments are fetched together into shared
+    // memory, so that a run crossing many short segments does not pay a chain of global
+    // round trips for each of them
+    __shared__ int64_t w_off[kSegWindow + 1];
+    __shared__ double w_piv[kSegWindow];
+    int w0 = -kSegWindow;  // first segment of the window (none loaded yet)
     while (cur < hi && s < S) {
-        const int64_t seg_end = off[s + 1];
+        if (s >= w0 + kSegWindow) {
+            __syncthreads();
+            w0 = s;
+            if (tid <= kSegWindow) w_off[tid] = off[(w0 + tid) <= S ? (w0 + tid) : S];
+            if (tid < kSegWindow) {
+                int64_t pi = off[(w0 + tid) < S ? (w0 + tid) : S - 1];
+                if (pi < 0 || pi >= d) pi = lo;
+                w_piv[tid] = (double)g[pi];  // the segment's pivot
+            }
+            __syncthreads();
+        }
+        const int64_t seg_end = w_off[s - w0 + 1];
         const int64_t sp_hi = seg_end < hi ? seg_end : hi;
         if (sp_hi > cur) {
             const Span sp = make_span(cur, sp_hi);
-            int64_t pi = off[s];
-            if (pi < 0 || pi >= d) pi = cur;
-            const double pv = (double)g[pi];  // the segment's pivot
+            const double pv = w_piv[s - w0];
             double sum = 0.0, sq = 0.0;
             // unaligned head and tail of the span: one element per thread
             const int nh = (int)(sp.a_lo - sp.lo), nt = (int)(sp.hi - sp.a_hi);
@@ -159,18 +192,20 @@ k_seg_accumulate_stats(const float* __restrict__ g, float* __restrict__ eps, int
             continue;
         }
         const int c0 = owner_cta(a, G, r4), c1 = owner_cta(b - 1, G, r4);
+        // the slots of one segment are added in ascending CTA order; loads go out sixteen at a
+        // time so that their latencies overlap
         double s1 = 0.0, s2 = 0.0;
-        for (int cc = c0; cc <= c1; ++cc) {
-            const double2 p = __ldcg(&v.partials[cc + q]);
-            s1 += p.x; s2 += p.y;
+        for (int cc = c0; cc <= c1; cc += 16) {
+            double2 p[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t)
+                p[t] = (cc + t <= c1) ? __ldcg(&v.partials[cc + t + q]) : make_double2(0.0, 0.0);
+#pragma unroll
+            for (int t = 0; t < 16; ++t) { s1 += p[t].x; s2 += p[t].y; }
         }
         int64_t kk = seg_k[q];
         if (kk > n) kk = n;
-        double zq = -INFINITY;
-        if (kk < n) {
-            const double p = 1.0 - (double)kk / (double)n;  // Algorithm 1: p = 1 - k/d
-            zq = normal_quantile_upper(1.0 - p);
-        }
+        const double zq = __ldcg(&v.zs[q]);
         alg1_thresholds(st, s1, s2, (double)g[a], n, kk, zq);
     }
     if (tid == 0) {
@@ -188,6 +223,7 @@ k_seg_count_candidates(const float* __restrict__ u, int64_t d, int64_t r4, const
                        const int64_t* __restrict__ seg_k, int S, Ctrl* __restrict__ ctrl, SegScratch v,
                        int64_t* __restrict__ seg_nnz_out) {
     __shared__ unsigned int s_cnt[kNumCand];
+    __shared__ int s_ord[kNumCand];
     __shared__ bool is_last;
     const int tid = threadIdx.x, c = blockIdx.x, G = gridDim.x;
     int64_t lo, hi;
@@ -196,46 +232,79 @@ k_seg_count_candidates(const float* __restrict__ u, int64_t d, int64_t r4, const
     const bool table_ok = (ctrl->stats.status & GK_DEV_BAD_SEGMENTS) == 0;
     int s = (lo < hi && table_ok) ? find_segment(off, S, lo) : S;
     int64_t cur = lo;
+    // per window of kSegWindow segments: end offsets, candidates in ascending order with their
+    // indices, and whether the segment needs counting at all; thread t prepares segment w0 + t
+    __shared__ int64_t w_end[kSegWindow];
+    __shared__ float w_cs[kSegWindow][kNumCand];
+    __shared__ unsigned char w_ord[kSegWindow][kNumCand];
+    __shared__ bool w_counted[kSegWindow];
+    int w0 = -kSegWindow;
     while (cur < hi && s < S) {
-        const int64_t seg_end = off[s + 1];
+        if (s >= w0 + kSegWindow) {
+            __syncthreads();
+            w0 = s;
+            if (tid < kSegWindow && w0 + tid < S) {
+                const int q = w0 + tid;
+                w_end[tid] = off[q + 1];
+                // segments that select everything need no counts
+                w_counted[tid] = v.stats[q].thr_final != -INFINITY;
+                float cd[kNumCand];
+                int od[kNumCand];
+#pragma unroll
+                for (int j = 0; j < kNumCand; ++j) cd[j] = v.cand32[(size_t)q * kNumCand + j];
+                for (int j = 0; j < kNumCand; ++j) {  // insertion sort of the ten thresholds
+                    int pos = j;
+                    while (pos > 0 && cd[od[pos - 1]] > cd[j]) { od[pos] = od[pos - 1]; --pos; }
+                    od[pos] = j;
+                }
+                for (int j = 0; j < kNumCand; ++j) { w_cs[tid][j] = cd[od[j]]; w_ord[tid][j] = (unsigned char)od[j]; }
+            }
+            __syncthreads();
+        }
+        const int ws = s - w0;
+        const int64_t seg_end = w_end[ws];
         const int64_t sp_hi = seg_end < hi ? seg_end : hi;
-        // segments that select everything (or nothing) need no counts
-        const bool counted = v.stats[s].thr_final != -INFINITY;
+        const bool counted = w_counted[ws];
         if (sp_hi > cur && counted) {
             const Span sp = make_span(cur, sp_hi);
-            if (tid < kNumCand) s_cnt[tid] = 0u;
-            float cand[kNumCand];
-            unsigned int cnt[kNumCand];
+            if (tid < kNumCand) { s_cnt[tid] = 0u; s_ord[tid] = w_ord[ws][tid]; }
+            __syncthreads();
+            float cs[kNumCand], acc[kNumCand];
 #pragma unroll
-            for (int j = 0; j < kNumCand; ++j) { cand[j] = v.cand32[(size_t)s * kNumCand + j]; cnt[j] = 0u; }
+            for (int j = 0; j < kNumCand; ++j) { cs[j] = w_cs[ws][j]; acc[j] = 0.f; }
+            const Tiers tier = make_tiers(cs);
+            const bool any_neg = cs[0] < 0.f;
             const int nh = (int)(sp.a_lo - sp.lo), nt = (int)(sp.hi - sp.a_hi);
             if (tid < nh || (tid >= 32 && tid < 32 + nt)) {
                 const float a = fabsf(u[tid < nh ? sp.lo + tid : sp.a_hi + (tid - 32)]);
 #pragma unroll
-                for (int j = 0; j < kNumCand; ++j) cnt[j] += (unsigned)(a > cand[j]);
+                for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
             }
+            // the warp's largest magnitude in each row of 32 float4 decides how many tiers to evaluate
             const int64_t i4_hi = sp.a_hi >> 2;
-            for (int64_t i4 = (sp.a_lo >> 2) + tid; i4 < i4_hi; i4 += 2 * kSegThreads) {
-                const int64_t j4 = i4 + kSegThreads;
-                const float4 x = __ldg(u4 + i4);
-                const float4 y = (j4 < i4_hi) ? __ldg(u4 + j4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                const float a0 = fabsf(x.x), a1 = fabsf(x.y), a2 = fabsf(x.z), a3 = fabsf(x.w);
-                const bool two = j4 < i4_hi;
-                const float b0 = fabsf(y.x), b1 = fabsf(y.y), b2 = fabsf(y.z), b3 = fabsf(y.w);
+            const int64_t i4_lo = sp.a_lo >> 2;
+            const int64_t n_it = (i4_hi - i4_lo + kSegThreads - 1) / kSegThreads;  // same for the whole warp
+            for (int64_t it = 0; it < n_it; it += 4) {
+                float4 x[4];
+                bool in[4];
 #pragma unroll
-                for (int j = 0; j < kNumCand; ++j) {
-                    cnt[j] += (unsigned)(a0 > cand[j]) + (unsigned)(a1 > cand[j]) + (unsigned)(a2 > cand[j]) +
-                              (unsigned)(a3 > cand[j]);
-                    if (two)
-                        cnt[j] += (unsigned)(b0 > cand[j]) + (unsigned)(b1 > cand[j]) + (unsigned)(b2 > cand[j]) +
-                                  (unsigned)(b3 > cand[j]);
+                for (int q = 0; q < 4; ++q) {
+                    const int64_t i4 = i4_lo + (it + q) * kSegThreads + tid;
+                    in[q] = i4 < i4_hi;
+                    x[q] = in[q] ? __ldg(u4 + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    unsigned int rm = (__reduce_max_sync(0xffffffffu, max_mag_bits(x[q])) + 0xffffu) >> 16;
+                    if (any_neg) rm = 0x10000u;
+                    if (in[q]) count_float4(x[q], rm, cs, tier, acc);
                 }
             }
             __syncthreads();
 #pragma unroll
             for (int j = 0; j < kNumCand; ++j) {
-                const unsigned int w = __reduce_add_sync(0xffffffffu, cnt[j]);
-                if ((tid & 31) == 0 && w) atomicAdd(&s_cnt[j], w);
+                const unsigned int w = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+                if ((tid & 31) == 0 && w) atomicAdd(&s_cnt[s_ord[j]], w);
             }
             __syncthreads();
             if (tid < kNumCand && s_cnt[tid]) {
@@ -288,20 +357,25 @@ extern "C" int gk_sparsify_segmented(const float* g, float* eps, int64_t d, cons
     const int n_tiles = (int)num_compact_tiles(d);
     // contiguous float4 runs of r4 per CTA, no CTA empty
     const int64_t n4 = d >> 2;
-    int64_t gmax = (int64_t)ws->sm_count * 4;
+    int64_t gmax = (int64_t)ws->sm_count * 2;  // two CTAs of 512 threads are resident per SM: one wave
     if (gmax > kMaxPartials) gmax = kMaxPartials;
     const int64_t min_run = 2 * kSegThreads;  // at least one full iteration per CTA
     int64_t r4 = (n4 + gmax - 1) / gmax;
     if (r4 < min_run) r4 = min_run;
     int64_t G = (n4 + r4 - 1) / r4;
     if (G < 1) G = 1;
+    stage_mark(ws, st, 0);
     k_seg_accumulate_stats<<<(int)G, kSegThreads, 0, st>>>(g, eps, d, r4, seg_offsets, seg_k, S, ws->ctrl, v,
                                                            ws->tile_status, n_tiles);
+    stage_mark(ws, st, 1);
     k_seg_count_candidates<<<(int)G, kSegThreads, 0, st>>>(eps, d, r4, seg_offsets, seg_k, S, ws->ctrl, v,
                                                            seg_nnz_out);
+    stage_mark(ws, st, 2);
     GK_CUDA_TRY(launch_compaction(k_compact_threshold<true>, n_tiles, ws->sm_count, st, eps, d, ws->ctrl,
                                   ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
                                   seg_offsets, (int)S, (const float*)v.thr_sel));
+    stage_mark(ws, st, 3);
+    ws->last_fused = false;
     note_launch(3);
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;

@@ -15,6 +15,7 @@ struct SegScratch {
     float* cand32;               // S x kNumCand
     float* thr_sel;              // S
     double2* partials;           // kMaxPartials + S: slot (cta + segment)
+    double* zs;                  // S: normal quantile of each segment's density
 };
 
 inline size_t seg_align(size_t x) { return (x + 255) / 256 * 256; }
@@ -28,6 +29,7 @@ inline size_t segmented_scratch_bytes(int64_t /*d*/, int32_t S) {
     at = seg_align(at + sizeof(float) * kNumCand * (size_t)S);
     at = seg_align(at + sizeof(float) * (size_t)S);
     at = seg_align(at + sizeof(double2) * ((size_t)kMaxPartials + (size_t)S));
+    at = seg_align(at + sizeof(double) * (size_t)S);
     return at;
 }
 
@@ -41,7 +43,8 @@ inline SegScratch segmented_views(const Workspace* ws) {
     v.counts = reinterpret_cast<unsigned long long*>(b + at);  at = seg_align(at + sizeof(unsigned long long) * kNumCand * S);
     v.cand32 = reinterpret_cast<float*>(b + at);               at = seg_align(at + sizeof(float) * kNumCand * S);
     v.thr_sel = reinterpret_cast<float*>(b + at);              at = seg_align(at + sizeof(float) * S);
-    v.partials = reinterpret_cast<double2*>(b + at);
+    v.partials = reinterpret_cast<double2*>(b + at);           at = seg_align(at + sizeof(double2) * ((size_t)kMaxPartials + S));
+    v.zs = reinterpret_cast<double*>(b + at);
     return v;
 }
 
