@@ -39,6 +39,10 @@ UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
 N_ROTATE = 20   # distinct gradients: the workload's 20 error-compensation iterations, then again
 EPISODE = 20    # steps that share one residual buffer (eps starts at zero)
+# DRAM bytes of one k_gk_fused launch at d = 25,557,032 (263.0 MB read + 77.4 MB written), from the
+# ncu capture summarised under profiles/; valid only for the kernel as it stood at that capture
+FUSED_DRAM_BYTES_PER_LAUNCH = 340418304
+FUSED_DRAM_CAPTURE_D = 25557032
 MAX_EPS = 48    # residual buffers kept (pre-zeroed); beyond that they are reused as they stand
 
 
@@ -296,7 +300,10 @@ def run_ours(args):
         "bound": "hbm", "kernel": "k_gk_fused", "achieved": bytes_step / (fused_ms * 1e-3) / 1e9,
         "peak": peak, "unit": "GB/s", "peak_source": peak_src,
         "frac": bytes_step / (fused_ms * 1e-3) / 1e9 / peak,
-        "traffic": None, "kernel_ms": fused_ms,
+        "traffic": FUSED_DRAM_BYTES_PER_LAUNCH if d == FUSED_DRAM_CAPTURE_D else None,
+        "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of k_gk_fused at this d "
+                          "(profiles/k_gk_fused_resnet50_ncu_full.txt)",
+        "kernel_ms": fused_ms,
         "phase_ms": {"accumulate_stats+barrier": fused[1], "count_loop": fused[2], "barrier2": fused[3],
                      "replay_rounds": fused[4], "compact": fused[5], "last_cta_exit": fused[6]},
         "bytes_per_launch": bytes_step,
