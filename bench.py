@@ -334,20 +334,44 @@ def run_ours(args):
         cold.append(a.elapsed_time(b))
     del flush
 
-    # ---- exact Top_k on the same data: operator (given u) and sparsifier (Eq. 2 with Top_k)
+    # ---- exact Top_k on the same data: operator (given u) and sparsifier (Eq. 2 with Top_k),
+    # as one cooperative kernel (path 0) and as histogram passes + look-back compaction (path 1)
     Kt = min(K, 100)
-    u = epss[0].clone()
+    us = [epss[j] for j in range(min(4, n_eps))]   # residual buffers of the loop above serve as u, in rotation
     tk_idx = torch.empty(k, dtype=torch.int32, device=dev)
     tk_val = torch.empty(k, dtype=torch.float32, device=dev)
-    for _ in range(3):
-        gk.topk_exact(u, k, tk_idx, tk_val)
-    ms_topk = time_region(torch, lambda t: gk.topk_exact(u, k, tk_idx, tk_val), Kt) / Kt
     eps2 = torch.zeros_like(epss[0])
-    for t in range(3):
-        gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz)
-    ms_topk_sp = time_region(torch, lambda t: gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz),
-                             Kt) / Kt
-    del eps2, u
+    topk = {}
+    for path, name in ((0, "fused"), (1, "multi_kernel")):
+        gk.gk_set_path(path)
+        for t in range(3):
+            gk.topk_exact(us[t % len(us)], k, tk_idx, tk_val)
+        ms_op = time_region(torch, lambda t: gk.topk_exact(us[t % len(us)], k, tk_idx, tk_val), Kt) / Kt
+        eps2.zero_()
+        for t in range(3):
+            gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz)
+        ms_sp = time_region(torch, lambda t: gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz),
+                            Kt) / Kt
+        rec = {"topk_exact_ms": ms_op, "topk_sparsify_ms": ms_sp,
+               "topk_exact_gbs_12B_per_elem": 12.0 * d / ms_op / 1e6,
+               "topk_sparsify_gbs_20B_per_elem": 20.0 * d / ms_sp / 1e6}
+        if path == 0:
+            gk.gk_stage_timing(True)
+            acc_op, acc_sp = np.zeros(8), np.zeros(8)
+            for t in range(20):
+                gk.topk_exact(us[t % len(us)], k, tk_idx, tk_val)
+                acc_op += np.array(gk.gk_last_stage_ms()[:8])
+                gk.topk_sparsify(gs[t % n_rot], eps2, k, tk_idx, tk_val, nnz)
+                acc_sp += np.array(gk.gk_last_stage_ms()[:8])
+            gk.gk_stage_timing(False)
+            names = ["kernel", "pass1", "barrier1+digit", "pass2+barrier2+digit", "pass3+barrier3+digit",
+                     "count+barrier4", "offsets+emit", "last_cta_exit"]
+            rec["phase_ms_operator"] = dict(zip(names, (acc_op / 20).tolist()))
+            rec["phase_ms_sparsifier"] = dict(zip(names, (acc_sp / 20).tolist()))
+        topk[name] = rec
+    gk.gk_set_path(0)
+    ms_topk, ms_topk_sp = topk["fused"]["topk_exact_ms"], topk["fused"]["topk_sparsify_ms"]
+    del eps2, us
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
     hg = [torch.from_numpy(w.grad(j, None)).pin_memory() for j in range(2)]
@@ -398,6 +422,7 @@ def run_ours(args):
         "topk": {"topk_exact_ms": ms_topk, "topk_sparsify_ms": ms_topk_sp,
                  "speedup_operator_vs_sparsifier": ms_topk / (ms / K),
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
+                 "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
         "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
         "clocks": sampler.summary(),

@@ -157,13 +157,14 @@ int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k, int32_t* 
  * is serving because that call stalls the whole device.  Same arguments, same
  * results and same capacity rule as gk_sparsify, but the call never reaches
  * cudaMalloc, cudaFree or any routine that allocates: its scratch is a fixed
- * 32 KB array inside the library image, present on every GPU that loads the
+ * 544 KB array inside the library image, present on every GPU that loads the
  * library for as long as the process lives.
  *
  * Limits: 1 <= k < d <= 2^31 - 1 (d beyond that returns GK_ERR_SIZE; k = d
  * returns GK_ERR_K: selecting everything is left to gk_sparsify); the device
- * must support cooperative launch and the launch must fit the array's 512
- * per-CTA slots, else GK_ERR_LIMIT.
+ * must support cooperative launch, the launch must fit the array's 512
+ * per-CTA slots, and the vector must not exceed 448 rows of 4096 elements per
+ * SM (271 M elements on 148 SMs), else GK_ERR_LIMIT.
  *
  * The first call on a device looks up the array's device address
  * (cudaGetSymbolAddress) and keeps it; make that first call before any stream

@@ -73,7 +73,8 @@ struct Workspace {
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
     unsigned int* cta_counts = nullptr;     // fused kernel: kFusedGridCap x kNumCand
-    unsigned int* bars = nullptr;           // fused kernel: two barrier counters and an exit counter
+    unsigned int* bars = nullptr;           // 16 counters: [0..2] barriers and exit of the fused sparsifier, [4..8] of the fused Top_k
+    unsigned int* rowcnt = nullptr;         // fused kernels: two words per row of 4096 elements
     unsigned long long* cta_trace = nullptr;  // fused kernel: kFusedGridCap x 8 timestamps (tracing aid)
     int last_grid = 0;                      // CTAs of the last fused launch
     // segmented call
@@ -83,6 +84,7 @@ struct Workspace {
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     int n_stages = 0;
     bool last_fused = false;  // the last sparsify call on this workspace ran the fused kernel
+    int phase_spans = 0;      // spans between the timestamps the last (single) kernel took itself; 0: none
 };
 
 // host side (gk_host.cu)
@@ -95,6 +97,8 @@ int64_t output_capacity(int64_t d);
 int selected_path();  // 0: fused kernel when usable, 1: three kernels with look-back
 int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                      float* val_out, int64_t* nnz_out, cudaStream_t st);
+int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                       float* val_out, int64_t* nnz_out, cudaStream_t st);
 int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                         float* val_out, int64_t* nnz_out, cudaStream_t st);
 

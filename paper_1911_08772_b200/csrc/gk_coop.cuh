@@ -1,0 +1,58 @@
+// Pieces shared by the persistent cooperative kernels (one CTA of 1024 threads
+// per SM, rows of 1024 float4): asynchronous copies, the L2-retaining store,
+// and the bounded grid barrier.  Internal.
+#pragma once
+
+#include "gk_common.cuh"
+
+namespace gk {
+
+constexpr int kFusedThreads = 1024;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kRowF4 = kFusedThreads;    // float4 per row
+constexpr int kRowBytes = kRowF4 * 16;   // 16 KB
+constexpr int kBarrierPollLimit = 1 << 24;
+
+#ifdef __CUDACC__
+
+// 16-byte asynchronous copy global -> shared, bypassing L1.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const unsigned int s = (unsigned int)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// 32-byte store that asks L2 to keep the line longer than ordinary traffic (the eviction
+// priority is only available on 256-bit accesses).  p must be 32-byte aligned.
+__device__ __forceinline__ void st_keep32(float4* p, const float4 a, const float4 b) {
+    asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(a.x), "f"(a.y),
+                 "f"(a.z), "f"(a.w), "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
+                 : "memory");
+}
+
+// Arrive at a barrier counter and wait until all G CTAs have arrived.
+// Returns false when the bounded wait ran out.
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int G, int* ok_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        int polls = 0;
+        bool ok = true;
+        while (true) {
+            unsigned int v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+            if (v >= G) break;
+            if (++polls > kBarrierPollLimit) { ok = false; break; }
+            __nanosleep(40);
+        }
+        *ok_flag = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *ok_flag != 0;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace gk

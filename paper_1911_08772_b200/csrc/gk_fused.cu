@@ -1,13 +1,14 @@
 // gk_sparsify as ONE persistent cooperative kernel (Eq. 2 and Algorithm 1 of
 // arXiv 1911.08772).
 //
-// One CTA per SM owns a contiguous run of the vector and streams through it in
-// rows of 1024 float4 (16 KB; thread t takes float4 t of the row).  The three
-// phases of the method are separated by two grid barriers, and what fits of u
-// stays on chip between them:
+// The vector is cut into rows of 1024 float4 (16 KB; thread t takes float4 t of
+// the row), dealt to one CTA per SM in turn (CTA c owns rows c, c + G, ...), so
+// that every CTA gets the same mix of the vector's quiet and loud stretches.
+// The three phases of the method are separated by grid barriers, and what fits
+// of u stays on chip between them:
 //
 //   phase A  g and eps arrive through a ring of asynchronous copies (cp.async,
-//            three rows ahead); u = g + eps is written over eps and into the
+//            kStages - 1 rows ahead); u = g + eps is written over eps and into the
 //            shared-memory slot its eps came through, so the last rows of the
 //            run are still on chip afterwards; fp64 partial sums per CTA; per
 //            (row, warp) the largest magnitude goes to a small table.
@@ -15,14 +16,14 @@
 //            mu, sigma, thres0 and the ten candidate thresholds for itself.
 //   phase B  counts of |u| > candidate for all ten candidates, from the
 //            on-chip copy where there is one, else from eps (L2 / HBM).
-//   barrier  every CTA reads all CTAs' counts, replays the rounds of
-//            Algorithm 1, and -- the count for the chosen threshold being
-//            known per CTA -- gets the output offset of its run directly.
-//            No look-back, no waiting between CTAs.
-//   phase C  groups of eight rows: a (row, warp) segment is read again only if
-//            its recorded maximum can exceed the threshold; an in-CTA scan
-//            orders the survivors; they are written as (index, value) pairs
-//            and their slots cleared.
+//   barrier  every CTA reads all CTAs' counts and replays the rounds of
+//            Algorithm 1: threshold and number of survivors are known.
+//   phase C  a (row, warp) segment is read again only if its recorded maximum
+//            can exceed the threshold; the survivors of every row are counted
+//            and the counts exchanged through a third barrier, which gives
+//            every row its output offset -- no look-back, no waiting between
+//            CTAs; the survivors are written as (index, value) pairs and
+//            their slots cleared.
 //
 // HBM traffic: 12 d bytes for phase A, 4 d for phase B on the rows that are not
 // on chip, and next to nothing for phase C (survivors are rare, so few segments
@@ -37,114 +38,79 @@
 
 #include "gk_alg1.cuh"
 #include "gk_common.cuh"
+#include "gk_coop.cuh"
 #include "gk_count.cuh"
 
 namespace gk {
 
-constexpr int kFusedThreads = 1024;
-constexpr int kFusedWarps = kFusedThreads / 32;
-constexpr int kRowF4 = kFusedThreads;                  // float4 per row
-constexpr int kRowBytes = kRowF4 * 16;                 // 16 KB
-constexpr int kTableMaxRows = 224;                     // rows beyond this are ordered in groups and always re-read
-constexpr int kTableBytes = kTableMaxRows * kFusedWarps * 2;  // 14 KB: one uint16 per (row, warp)
-constexpr int kSmemRows = 13;                          // 16 KB rows of dynamic shared memory
-constexpr int kFusedSmemBytes = kSmemRows * kRowBytes + kTableBytes;  // ring, u slots, table
+constexpr int kTableMaxRows = 448;                     // most rows a CTA may own (entries of its maximum table)
+constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
+constexpr int kFusedSmemBudget = 226304;               // dynamic shared memory the kernel may ask for
 constexpr int kStages = 4;                             // phase A: rows of g and eps in flight, plus one
 constexpr int kRing = 8;                               // ring slots; phase B has kRing - 1 rows in flight
-constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
-constexpr int kGroupRows = 8;                          // rows ordered by one in-CTA scan
+constexpr int kGroupRows = 8;                          // rows a warp gathers per batch in phase C
 constexpr int kFusedMaxGrid = kFusedGridCap;
-constexpr int kBarrierPollLimit = 1 << 24;
 constexpr int kTraceSlots = 8;                         // timestamps per CTA in the optional trace
 
-struct FusedShared {
+struct __align__(128) FusedShared {
     double2 red[kFusedWarps];
     unsigned int cta_counts[kNumCand];
     unsigned long long col[kNumCand];   // counts over the whole vector
-    unsigned long long colpre[kNumCand];  // counts over the runs of the CTAs before this one
     double cand64[kNumCand];
     float cand32[kNumCand];
     int order[kNumCand];                // candidate indices, ascending by threshold
     float thr_sel;
     int chosen;
     int ok;
-    unsigned long long base;            // survivors in earlier CTAs
     gk_stats stats;
-    // ordering scan of one group of rows
-    unsigned int wtot[kGroupRows][kFusedWarps];
-    unsigned int woff[kGroupRows][kFusedWarps];
-    unsigned int rtot[kGroupRows];
-    unsigned int rowpre[kTableMaxRows];  // survivors in the rows before each row of this CTA
+    unsigned int wsum[kFusedWarps];
+    unsigned int roundtot[kTableMaxRows];  // survivors in each round of rows (G consecutive rows)
+    unsigned int rowpre[kTableMaxRows];    // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
 };
 
-// 16-byte asynchronous copy global -> shared, bypassing L1.
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    const unsigned int s = (unsigned int)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// 32-byte store that asks L2 to keep the line longer than ordinary traffic (the eviction
-// priority is only available on 256-bit accesses).  p must be 32-byte aligned.
-__device__ __forceinline__ void st_keep32(float4* p, const float4 a, const float4 b) {
-    asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(a.x), "f"(a.y),
-                 "f"(a.z), "f"(a.w), "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
-                 : "memory");
-}
-
-// Arrive at a barrier counter and wait until all G CTAs have arrived.
-// Returns false when the bounded wait ran out.
-__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int G, int* ok_flag) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(counter, 1u);
-        int polls = 0;
-        bool ok = true;
-        while (true) {
-            unsigned int v;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-            if (v >= G) break;
-            if (++polls > kBarrierPollLimit) { ok = false; break; }
-            __nanosleep(40);
-        }
-        *ok_flag = ok ? 1 : 0;
-    }
-    __syncthreads();
-    return *ok_flag != 0;
-}
+static_assert((sizeof(FusedShared) + 1023) / 1024 * 1024 + kFusedSmemBudget <= 232448,
+              "over the 227 KB of shared memory per CTA (the dynamic part starts on a 1 KB boundary)");
 
 __device__ __forceinline__ unsigned int mask_above(const float4 v, const float thr) {
     return (unsigned)(fabsf(v.x) > thr) | ((unsigned)(fabsf(v.y) > thr) << 1) |
            ((unsigned)(fabsf(v.z) > thr) << 2) | ((unsigned)(fabsf(v.w) > thr) << 3);
 }
 
-// rows_per_cta: rows of the run of every CTA; u_slots: row slots of shared memory
-// that receive eps and then hold u (the last u_slots rows of the run stay on
-// chip); table_rows: rows that have an entry in the maximum table.
-// Shared memory: [ring of kRing rows][u_slots rows][table].
+// n_rows: rows of 1024 float4 in the whole vector; CTA c owns rows c, c + G, c + 2G, ...
+// (G = gridDim.x), so that stretches of large values are spread over all CTAs.  u_slots: row
+// slots of shared memory that receive eps and then hold u (the last u_slots rows of a CTA stay
+// on chip); table_rows: the largest number of rows any CTA owns (entries of the maximum table).
+// rowcnt: one word per row of the vector.
+// Shared memory: [ring of kRing rows][u_slots rows][table of table_rows x 32 uint16].
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
-           int rows_per_cta, int u_slots, int table_rows, Ctrl* __restrict__ ctrl,
+           int n_rows, int u_slots, int table_rows, Ctrl* __restrict__ ctrl,
            double2* __restrict__ partials, unsigned int* __restrict__ cta_counts,
-           unsigned int* __restrict__ bars, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
-           int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
-    extern __shared__ float4 smem4[];
+           unsigned int* __restrict__ bars, unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out,
+           float* __restrict__ val_out, int64_t* __restrict__ nnz_out, int64_t cap,
+           unsigned long long* __restrict__ trace) {
+    // 1 KB alignment keeps every warp's 512 bytes of a row within four 128-byte lines of shared
+    // memory, whatever the size of the static part
+    extern __shared__ __align__(1024) float4 smem4[];
     __shared__ FusedShared sh;
     float4* gring = smem4;                                   // kRing x kRowF4 (phase A uses kStages of them)
     float4* uslot = smem4 + (size_t)kRing * kRowF4;          // u_slots x kRowF4
-    unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)kSmemRows * kRowF4);
+    unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)(kRing + u_slots) * kRowF4);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int c = blockIdx.x, G = gridDim.x;
     const int64_t n4 = d >> 2;
 
-    // this CTA's run of float4
-    int64_t lo4 = (int64_t)c * rows_per_cta * kRowF4, hi4 = lo4 + (int64_t)rows_per_cta * kRowF4;
-    if (lo4 > n4) lo4 = n4;
-    if (hi4 > n4) hi4 = n4;
-    const int nrows = (int)((hi4 - lo4 + kRowF4 - 1) / kRowF4);
+    // this CTA's rows: local row r is row c + r * G of the vector; only the last row of the
+    // vector can be short, and it is the last local row of the CTA that owns it
+    const int nrows = c < n_rows ? (n_rows - c + G - 1) / G : 0;
+    const int64_t stride4 = (int64_t)G * kRowF4;             // from a local row to the next
+    const int64_t first4 = (int64_t)c * kRowF4 + tid;        // this thread's float4 in local row 0
+    const bool has_last = nrows > 0 && (c + (nrows - 1) * G == n_rows - 1);
+    const bool in_last_row = !(has_last && (n4 & (kRowF4 - 1)) != 0) || tid < (int)(n4 & (kRowF4 - 1));
+    // rows from first_kept on stay on chip after phase A; the short last row of the vector, if
+    // this CTA owns it, is its last row and therefore among them (u_slots >= 1)
+    const int first_kept = nrows > u_slots ? nrows - u_slots : 0;
     const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
     const int64_t tail_i = (n4 << 2) + lane;
     const float4* g4 = reinterpret_cast<const float4*>(g);
@@ -167,21 +133,22 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
         // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
         // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
+        int64_t fi = first4;  // the row the next fetch brings in
         auto fetch = [&](int r) {
-            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-            if (r < nrows && i < hi4) {
-                cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + i);
-                cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + i);
+            if (r < nrows && fi < n4) {
+                cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
+                cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + fi);
             }
             cp_async_commit();
+            fi += stride4;
         };
 #pragma unroll
         for (int r = 0; r < kStages - 1; ++r) fetch(r);
-        for (int r = 0; r < nrows; ++r) {
+        int64_t i = first4;
+        for (int r = 0; r < nrows; ++r, i += stride4) {
             fetch(r + kStages - 1);
             cp_async_wait<kStages - 1>();
-            const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-            const bool one = i < hi4;
+            const bool one = i < n4;
             float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one) {
                 float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
@@ -199,7 +166,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 float4 nb;
                 nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
                 nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
-                const bool pair = wide_ok && (i + 1 < hi4);  // this lane and its right neighbour are in range
+                const bool pair = wide_ok && (i + 1 < n4);  // this lane and its right neighbour are in range
                 if ((lane & 1) == 0) {
                     if (pair) st_keep32(e4 + i, u0, nb);
                     else if (one) e4[i] = u0;
@@ -209,7 +176,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             }
             // largest magnitude of each (row, warp) segment, top 16 bits rounded up
             const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
-            if (lane == 0 && r < table_rows) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
+            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
         }
         cp_async_wait<0>();
         if (owns_tail) {
@@ -263,21 +230,17 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         tier.t7 = __float_as_uint(fmaxf(cs[7], 0.f)) >> 16;
         const unsigned int always = 0x10000u;  // above every 16-bit maximum
         const bool any_neg = cs[0] < 0.f;
-        const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
-        // only the last row of a run can be short: `mine_last` says whether this thread has a part in it
-        const int nfull = (int)((hi4 - lo4) / kRowF4);
-        const bool mine_last = lo4 + (int64_t)nfull * kRowF4 + tid < hi4;
-        const float4* src = e4 + lo4 + tid;
         const unsigned short* trow = table + w;
         // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
-        // in phase A, kRing - 1 rows ahead of the counting
+        // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows
+        const float4* fp = e4 + first4;  // the row the next fetch brings in
         auto fetch_u = [&](int r) {
-            if (r < first_kept && (r < nfull || mine_last))
-                cp_async16(gring + ((r & (kRing - 1)) << 10) + tid, src + ((size_t)r << 10));
+            if (r < first_kept) cp_async16(gring + ((r & (kRing - 1)) << 10) + tid, fp);
             cp_async_commit();
+            fp += stride4;
         };
         auto row_max = [&](int r) -> unsigned int {
-            return (any_neg || r >= table_rows) ? always : (unsigned int)trow[r * kFusedWarps];
+            return any_neg ? always : (unsigned int)trow[r * kFusedWarps];
         };
 #pragma unroll
         for (int r = 0; r < kRing - 1; ++r) fetch_u(r);
@@ -287,12 +250,11 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         for (; r < first_kept; ++r) {
             fetch_u(r + kRing - 1);
             cp_async_wait<kRing - 1>();
-            if (r < nfull || mine_last)
-                count_float4(gring[((r & (kRing - 1)) << 10) + tid], row_max(r), cs, tier, acc);
+            count_float4(gring[((r & (kRing - 1)) << 10) + tid], row_max(r), cs, tier, acc);
         }
         cp_async_wait<0>();
         for (r = first_kept; r < nrows; ++r) {
-            if (r < nfull || mine_last)
+            if (r != nrows - 1 || in_last_row)
                 count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], row_max(r), cs, tier, acc);
         }
         if (owns_tail) {
@@ -319,8 +281,8 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
 
     // ------------------------------------------------------------------ resolve
     {
-        // warp j adds column j over all CTAs and, separately, over the CTAs before this one
-        // (integer sums: the order does not matter); the loads are independent of each other
+        // warp j adds column j over all CTAs (integer sums: the order does not matter); the loads
+        // are independent of each other
         if (w < kNumCand) {
             unsigned int v[kFusedMaxGrid / 32];
 #pragma unroll
@@ -328,34 +290,32 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 const int t = lane + 32 * q;
                 v[q] = (t < G) ? __ldcg(&cta_counts[(size_t)t * kNumCand + w]) : 0u;
             }
-            unsigned long long s = 0ull, pre = 0ull;
+            unsigned long long s = 0ull;
 #pragma unroll
-            for (int q = 0; q < kFusedMaxGrid / 32; ++q) {
-                s += v[q];
-                if (lane + 32 * q < c) pre += v[q];
-            }
+            for (int q = 0; q < kFusedMaxGrid / 32; ++q) s += v[q];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                s += __shfl_xor_sync(0xffffffffu, s, o);
-                pre += __shfl_xor_sync(0xffffffffu, pre, o);
-            }
-            if (lane == 0) { sh.col[w] = s; sh.colpre[w] = pre; }
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) sh.col[w] = s;
         }
         __syncthreads();
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
             sh.chosen = alg1_resolve(st, k);
-            sh.base = sh.colpre[sh.chosen];
         }
         __syncthreads();
         if (c == 0 && tid == 0) {
             const long long all = sh.stats.nnz;
             const long long written = all < cap ? all : cap;
-            sh.stats.emitted = written;
-            if (all > cap) sh.stats.status |= GK_DEV_TRUNCATED;
-            const int late = ctrl->stats.status & GK_DEV_TIMEOUT;
-            ctrl->stats = sh.stats;
-            if (late) atomicOr(&ctrl->stats.status, late);
+            // every field but the status word, which was cleared at the start and only ever has
+            // flags added to it (a CTA that gave up waiting may have added one already)
+            gk_stats* o = &ctrl->stats;
+            o->mu = sh.stats.mu; o->sigma = sh.stats.sigma; o->z = sh.stats.z;
+            o->thres0 = sh.stats.thres0; o->thr_final = sh.stats.thr_final;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) o->counts[j] = sh.stats.counts[j];
+            o->rounds = sh.stats.rounds; o->nnz = all; o->emitted = written;
+            const int flags = sh.stats.status | (all > cap ? GK_DEV_TRUNCATED : 0);
+            if (flags) atomicOr(&o->status, flags);
             *nnz_out = written;
             ctrl->phase_t[4] = global_timer_ns();
         }
@@ -363,48 +323,51 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     }
 
     // ------------------------------------------------------------------ phase C
-    {
+    // The survivor count of the whole vector is known to every CTA; with none there is nothing
+    // left to do (the same decision in every CTA, so the barrier below is reached by all or none).
+    if (sh.stats.nnz != 0) {
         const float thr = sh.thr_sel;
-        const unsigned int mine = sh.cta_counts[sh.chosen];  // survivors in this CTA's run
+        const unsigned int mine = sh.cta_counts[sh.chosen];  // survivors in this CTA's rows
         // a segment can hold a survivor only if its recorded maximum (rounded up to 16 bits)
         // exceeds the threshold's top 16 bits; a negative threshold admits everything
         const bool all_pass = thr < 0.0f;
         const unsigned int thr16 = __float_as_uint(fmaxf(thr, 0.0f)) >> 16;
-        unsigned long long run = sh.base;
-        const int trows = nrows < table_rows ? nrows : table_rows;  // rows covered by the table
-        const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on are on chip
+        constexpr unsigned short kPending = 0xffffu;
+        // up to kGroupRows rows of this warp whose entry is pending (want_pending) or non-zero,
+        // from `cursor` on
+        auto gather = [&](int& cursor, const bool want_pending) -> int {
+            int n = 0;
+            while (n < kGroupRows && cursor < nrows) {
+                const int r = cursor + lane;
+                unsigned int e = 0u;
+                if (r < nrows) e = table[r * kFusedWarps + w];
+                const bool hit = want_pending ? (e == kPending) : (e != 0u);
+                unsigned int b = __ballot_sync(0xffffffffu, hit);
+                while (b && n < kGroupRows) {
+                    const int bit = __ffs(b) - 1;
+                    if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
+                    ++n;
+                    b &= b - 1u;
+                }
+                if (b) { cursor += __ffs(b) - 1; break; }
+                cursor += 32;
+            }
+            __syncwarp();
+            return n;
+        };
+        auto load_row = [&](int r, int64_t i) -> float4 {
+            return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
+        };
         if (mine != 0u) {
             // step 1: every warp counts the survivors of its qualifying segments; the table
             // entry of a segment is replaced by that count (0 where it cannot qualify).
             // Qualifying rows are gathered eight at a time so that their loads overlap.
-            constexpr unsigned short kPending = 0xffffu;
-            for (int r = lane; r < trows; r += 32) {
+            for (int r = lane; r < nrows; r += 32) {
                 const bool ql = all_pass || table[r * kFusedWarps + w] > thr16;
                 table[r * kFusedWarps + w] = ql ? kPending : (unsigned short)0;
             }
             __syncwarp();
-            // up to kGroupRows rows of this warp whose entry satisfies want(entry), from `cursor` on
-            auto gather = [&](int& cursor, const bool want_pending) -> int {
-                int n = 0;
-                while (n < kGroupRows && cursor < trows) {
-                    const int r = cursor + lane;
-                    unsigned int e = 0u;
-                    if (r < trows) e = table[r * kFusedWarps + w];
-                    const bool hit = want_pending ? (e == kPending) : (e != 0u);
-                    unsigned int b = __ballot_sync(0xffffffffu, hit);
-                    while (b && n < kGroupRows) {
-                        const int bit = __ffs(b) - 1;
-                        if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
-                        ++n;
-                        b &= b - 1u;
-                    }
-                    if (b) { cursor += __ffs(b) - 1; break; }
-                    cursor += 32;
-                }
-                __syncwarp();
-                return n;
-            };
-            for (int cursor = 0; cursor < trows;) {
+            for (int cursor = 0; cursor < nrows;) {
                 const int n = gather(cursor, true);
                 float4 v[kGroupRows];
 #pragma unroll
@@ -412,60 +375,86 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (q < n) {
                         const int r = sh.qrow[w][q];
-                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                        if (i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
+                        const int64_t i = (first4 + (int64_t)r * stride4);
+                        if (i < n4) v[q] = load_row(r, i);
                     }
                 }
 #pragma unroll
                 for (int q = 0; q < kGroupRows; ++q) {
                     if (q < n) {
                         const int r = sh.qrow[w][q];
-                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+                        const int64_t i = (first4 + (int64_t)r * stride4);
                         const unsigned int cnt =
-                            __reduce_add_sync(0xffffffffu, i < hi4 ? __popc(mask_above(v[q], thr)) : 0u);
+                            __reduce_add_sync(0xffffffffu, i < n4 ? __popc(mask_above(v[q], thr)) : 0u);
                         if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
                     }
                 }
                 __syncwarp();
             }
-            __syncthreads();
-            // step 2: survivors per row, exclusive scan over the rows (thread t takes row t)
-            {
-                unsigned int mine_row = 0u;
-                if (tid < trows) {
-                    const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
+        }
+        __syncthreads();
+        // step 2: survivors per row (thread t takes local row t) go to the row's word in global
+        // memory; every row of the vector gets its word from the CTA that owns it
+        if (tid < nrows) {
+            unsigned int mine_row = 0u;
+            if (mine != 0u) {
+                const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
 #pragma unroll
-                    for (int q = 0; q < kTableRowBytes / 16; ++q) {
-                        const uint4 x = tv[q];
-                        mine_row += (x.x & 0xffffu) + (x.x >> 16) + (x.y & 0xffffu) + (x.y >> 16) +
-                                    (x.z & 0xffffu) + (x.z >> 16) + (x.w & 0xffffu) + (x.w >> 16);
-                    }
+                for (int q = 0; q < kTableRowBytes / 16; ++q) {
+                    const uint4 x = tv[q];
+                    mine_row += (x.x & 0xffffu) + (x.x >> 16) + (x.y & 0xffffu) + (x.y >> 16) +
+                                (x.z & 0xffffu) + (x.z >> 16) + (x.w & 0xffffu) + (x.w >> 16);
                 }
-                unsigned int s = mine_row;
+            }
+            rowcnt[c + tid * G] = mine_row;
+        }
+        stamp(5);
+        if (!grid_barrier(&bars[3], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        stamp(6);
+        if (mine != 0u) {
+            // Survivors before local row r of this CTA = those of the rounds before r (round r is
+            // the G consecutive rows r * G ... r * G + G - 1) + those of the CTAs before this one
+            // in round r.  Warp j takes rounds j, j + 32, ...
+            for (int r = w; r < nrows; r += kFusedWarps) {
+                unsigned int tot = 0u, pre = 0u;
+                const int R0 = r * G;
+                for (int t = lane; t < G; t += 32) {
+                    const unsigned int v = (R0 + t < n_rows) ? __ldcg(rowcnt + R0 + t) : 0u;
+                    tot += v;
+                    pre += (t < c) ? v : 0u;
+                }
+                tot = __reduce_add_sync(0xffffffffu, tot);
+                pre = __reduce_add_sync(0xffffffffu, pre);
+                if (lane == 0) { sh.roundtot[r] = tot; sh.rowpre[r] = pre; }
+            }
+            __syncthreads();
+            // exclusive scan of the round totals (thread t takes round t; at most kTableMaxRows)
+            {
+                const unsigned int mine_round = tid < nrows ? sh.roundtot[tid] : 0u;
+                unsigned int s = mine_round;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const unsigned int t = __shfl_up_sync(0xffffffffu, s, o);
                     if (lane >= o) s += t;
                 }
-                if (lane == 31) sh.wtot[0][w] = s;
+                if (lane == 31) sh.wsum[w] = s;
                 __syncthreads();
-                if (w == 0) {
-                    const unsigned int x = sh.wtot[0][lane];
-                    unsigned int y = x;
+                const unsigned int x = sh.wsum[lane];
+                unsigned int y = x;
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const unsigned int t = __shfl_up_sync(0xffffffffu, y, o);
-                        if (lane >= o) y += t;
-                    }
-                    sh.woff[0][lane] = y - x;
-                    if (lane == 31) sh.rtot[0] = y;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int t = __shfl_up_sync(0xffffffffu, y, o);
+                    if (lane >= o) y += t;
                 }
-                __syncthreads();
-                if (tid < trows) sh.rowpre[tid] = sh.woff[0][w] + s - mine_row;
+                const unsigned int wpre = __shfl_sync(0xffffffffu, y - x, w);
+                if (tid < nrows) sh.rowpre[tid] += wpre + s - mine_round;
                 __syncthreads();
             }
             // step 3: every warp writes the survivors of its segments that have any
-            for (int cursor = 0; cursor < trows;) {
+            for (int cursor = 0; cursor < nrows;) {
                 const int n = gather(cursor, false);
                 float4 v[kGroupRows];
 #pragma unroll
@@ -473,16 +462,16 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (q < n) {
                         const int r = sh.qrow[w][q];
-                        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                        if (i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
+                        const int64_t i = (first4 + (int64_t)r * stride4);
+                        if (i < n4) v[q] = load_row(r, i);
                     }
                 }
 #pragma unroll
                 for (int q = 0; q < kGroupRows; ++q) {
                     if (q >= n) continue;
                     const int r = sh.qrow[w][q];
-                    const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                    const unsigned int m = i < hi4 ? mask_above(v[q], thr) : 0u;
+                    const int64_t i = (first4 + (int64_t)r * stride4);
+                    const unsigned int m = i < n4 ? mask_above(v[q], thr) : 0u;
                     // survivors of this row in the warps before this one
                     const unsigned int before =
                         __reduce_add_sync(0xffffffffu, lane < w ? (unsigned int)table[r * kFusedWarps + lane] : 0u);
@@ -494,13 +483,13 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                         if (lane >= o) sc += t;
                     }
                     if (m) {
-                        unsigned long long p = run + sh.rowpre[r] + before + (sc - c_m);
+                        long long p = (long long)sh.rowpre[r] + before + (sc - c_m);
                         const int64_t e0 = i << 2;
                         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
                             if (m & (1u << t)) {
-                                if ((long long)p < cap) {
+                                if (p < cap) {
                                     idx_out[p] = (int32_t)(e0 + t);
                                     val_out[p] = vv[t];
                                     eps[e0 + t] = 0.0f;
@@ -512,102 +501,14 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 }
                 __syncwarp();
             }
-            run += sh.rtot[0];
-            __syncthreads();  // the scan arrays are reused below
-            // rows beyond the table (vectors of more than ~230 M elements): ordered in groups
-            for (int r0 = trows; r0 < nrows; r0 += kGroupRows) {
-                // does any segment of this group qualify?  (the same answer in every warp)
-                bool any = all_pass;
-                if (!any) {
-#pragma unroll
-                    for (int q = 0; q < kGroupRows; ++q) {
-                        const int r = r0 + q;
-                        if (r < nrows) any |= (r >= table_rows) || (table[r * kFusedWarps + lane] > thr16);
-                    }
-                    any = __any_sync(0xffffffffu, any);
-                }
-                if (!any) continue;
-                float4 v[kGroupRows];
-                unsigned int m[kGroupRows];
-#pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    const int r = r0 + q;
-                    const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    m[q] = 0u;
-                    // warp-uniform: skip the segment when its maximum cannot pass
-                    const bool look = r < nrows &&
-                                      (all_pass || r >= table_rows || table[r * kFusedWarps + w] > thr16);
-                    if (look && i < hi4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
-                }
-#pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    const int64_t i = lo4 + (int64_t)(r0 + q) * kRowF4 + tid;
-                    if (r0 + q < nrows && i < hi4) m[q] = mask_above(v[q], thr);
-                }
-                // order: (row, warp, lane).  Packed byte scans inside the warp, then over warps.
-                unsigned int incl[kGroupRows / 4];
-#pragma unroll
-                for (int h = 0; h < kGroupRows / 4; ++h) {
-                    unsigned int p = __popc(m[4 * h]) | (__popc(m[4 * h + 1]) << 8) | (__popc(m[4 * h + 2]) << 16) |
-                                     (__popc(m[4 * h + 3]) << 24);
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const unsigned int t = __shfl_up_sync(0xffffffffu, p, o);
-                        if (lane >= o) p += t;  // bytes hold at most 32 * 4 = 128
-                    }
-                    incl[h] = p;
-                    if (lane == 31) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) sh.wtot[4 * h + q][w] = (p >> (8 * q)) & 0xffu;
-                    }
-                }
-                __syncthreads();
-                if (w < kGroupRows) {
-                    const unsigned int x = sh.wtot[w][lane];
-                    unsigned int s = x;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const unsigned int t = __shfl_up_sync(0xffffffffu, s, o);
-                        if (lane >= o) s += t;
-                    }
-                    sh.woff[w][lane] = s - x;
-                    if (lane == 31) sh.rtot[w] = s;
-                }
-                __syncthreads();
-                unsigned long long row_base = run;
-#pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    if (m[q]) {
-                        const unsigned int c_q = __popc(m[q]);
-                        unsigned long long p = row_base + sh.woff[q][w] + ((incl[q >> 2] >> (8 * (q & 3))) & 0xffu) - c_q;
-                        const int64_t e0 = (lo4 + (int64_t)(r0 + q) * kRowF4 + tid) << 2;
-                        const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            if (m[q] & (1u << t)) {
-                                if ((long long)p < cap) {
-                                    idx_out[p] = (int32_t)(e0 + t);
-                                    val_out[p] = vv[t];
-                                    eps[e0 + t] = 0.0f;
-                                }
-                                ++p;
-                            }
-                        }
-                    }
-                    row_base += sh.rtot[q];
-                }
-                run = row_base;
-                __syncthreads();  // the scan arrays are reused by the next group
-            }
         }
         // the ragged tail comes last in index order
         if ((c == G - 1) && (w == kFusedWarps - 1) && (d & 3)) {
             const bool hit = owns_tail && (fabsf(tail_u) > thr);
             const unsigned int bal = __ballot_sync(0xffffffffu, hit);
             if (hit) {
-                const unsigned long long p = run + __popc(bal & ((1u << lane) - 1u));
-                if ((long long)p < cap) {
+                const long long p = (long long)sh.stats.nnz - __popc(bal) + __popc(bal & ((1u << lane) - 1u));
+                if (p < cap) {
                     idx_out[p] = (int32_t)tail_i;
                     val_out[p] = tail_u;
                     eps[tail_i] = 0.0f;
@@ -617,7 +518,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     }
 
     if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
-    stamp(5);
+    stamp(7);
 
 leave:
     // the CTA that leaves last clears the barrier counters for the next call
@@ -627,7 +528,7 @@ leave:
         const unsigned int t = atomicAdd(&bars[2], 1u);
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[6] = global_timer_ns();
-            bars[0] = 0u; bars[1] = 0u;
+            bars[0] = 0u; bars[1] = 0u; bars[3] = 0u;
             __threadfence();
             bars[2] = 0u;
         }
@@ -648,13 +549,13 @@ static FusedPlan* fused_plan(int dev, int sm_count) {
     p.ready = true;
     int coop = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return &p;
-    if (cudaFuncSetAttribute(k_gk_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBytes) !=
+    if (cudaFuncSetAttribute(k_gk_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBudget) !=
         cudaSuccess) {
         cudaGetLastError();
         return &p;
     }
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused, kFusedThreads, kFusedSmemBytes) !=
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused, kFusedThreads, kFusedSmemBudget) !=
             cudaSuccess || occ < 1) {
         cudaGetLastError();
         return &p;
@@ -666,38 +567,45 @@ static FusedPlan* fused_plan(int dev, int sm_count) {
 
 // Launch geometry for a vector of d elements on a grid of at most `grid` CTAs.
 struct FusedGeometry {
-    int64_t G;       // CTAs (none without rows)
-    int rpc;         // rows per CTA
+    bool fits;       // false: a CTA would own more rows than its table holds
+    int64_t G;       // CTAs (none without rows, at least one)
+    int n_rows;      // rows of 1024 float4 in the vector
     int u_slots;     // row slots of shared memory that end up holding u
-    int table_rows;  // rows with an entry in the maximum table
+    int table_rows;  // the largest number of rows a CTA owns
+    size_t smem;     // dynamic shared memory of the launch
 };
 static FusedGeometry fused_geometry(int64_t d, int grid) {
     FusedGeometry q;
     const int64_t n4 = d >> 2;
-    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;  // rows in the whole vector
-    int64_t rows_per_cta = (n_rows + grid - 1) / grid;
-    if (rows_per_cta < 1) rows_per_cta = 1;
-    q.G = (n_rows + rows_per_cta - 1) / rows_per_cta;
+    const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;
+    q.n_rows = (int)n_rows;
+    q.G = n_rows < grid ? n_rows : grid;
     if (q.G < 1) q.G = 1;
-    q.rpc = (int)rows_per_cta;
-    // shared memory: the g ring and the maximum table claim their share, the rest holds u
-    q.table_rows = q.rpc < kTableMaxRows ? q.rpc : kTableMaxRows;
-    q.u_slots = kSmemRows - kRing;
-    if (q.u_slots > q.rpc) q.u_slots = q.rpc;
+    int64_t most = (n_rows + q.G - 1) / q.G;  // rows of CTA 0
+    if (most < 1) most = 1;
+    q.fits = most <= kTableMaxRows;
+    q.table_rows = (int)(most < kTableMaxRows ? most : kTableMaxRows);
+    // shared memory: the ring and the maximum table claim their share, the rest holds u
+    const int64_t left = (int64_t)kFusedSmemBudget - (int64_t)kRing * kRowBytes - (int64_t)q.table_rows * kTableRowBytes;
+    q.u_slots = (int)(left / kRowBytes);
+    if (q.u_slots > most) q.u_slots = (int)most;
+    if (q.u_slots < 1) q.fits = false;
+    q.smem = (size_t)(kRing + q.u_slots) * kRowBytes + (size_t)q.table_rows * kTableRowBytes;
     return q;
 }
 
 // The one place that builds the kernel's argument list (types checked by the compiler).
-static cudaError_t launch_fused(int64_t G, cudaStream_t st, const float* g, float* eps, int64_t d, int64_t k, double z,
-                                int rpc, int u_slots, int table_rows, Ctrl* ctrl, double2* partials,
-                                unsigned int* cta_counts, unsigned int* bars, int32_t* idx_out, float* val_out,
+static cudaError_t launch_fused(const FusedGeometry& geo, cudaStream_t st, const float* g, float* eps, int64_t d,
+                                int64_t k, double z, Ctrl* ctrl, double2* partials, unsigned int* cta_counts,
+                                unsigned int* bars, unsigned int* rowcnt, int32_t* idx_out, float* val_out,
                                 int64_t* nnz_out, int64_t cap, unsigned long long* trace) {
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&rpc, (void*)&u_slots,
+    int n_rows = geo.n_rows, u_slots = geo.u_slots, table_rows = geo.table_rows;
+    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&n_rows, (void*)&u_slots,
                     (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
-                    (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap, (void*)&trace};
-    static_assert(sizeof(args) / sizeof(args[0]) == 17, "k_gk_fused takes 17 arguments");
-    return cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)G), dim3(kFusedThreads), args,
-                                       (size_t)kFusedSmemBytes, st);
+                    (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap, (void*)&trace};
+    static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused takes 18 arguments");
+    return cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)geo.G), dim3(kFusedThreads), args,
+                                       geo.smem, st);
 }
 
 // Returns GK_OK when the fused kernel was enqueued, 1 when it cannot be used on
@@ -709,24 +617,18 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
     GK_CUDA_TRY(cudaGetDevice(&dev));
     FusedPlan* p = fused_plan(dev, ws->sm_count);
     if (!p || !p->usable || k >= d) return 1;
-    FusedGeometry geo = fused_geometry(d, p->grid);
-    int64_t G = geo.G;
-    int rpc = geo.rpc, u_slots = geo.u_slots, table_rows = geo.table_rows;
+    const FusedGeometry geo = fused_geometry(d, p->grid);
+    if (!geo.fits) return 1;
     const double pq = 1.0 - (double)k / (double)d;  // Algorithm 1: p = 1 - k/d
-    double z = normal_quantile_upper(1.0 - pq);
-    int64_t cap = output_capacity(d);
-    Ctrl* ctrl = ws->ctrl;
-    double2* partials = ws->partials;
-    unsigned int* cta_counts = ws->cta_counts;
-    unsigned int* bars = ws->bars;
-    unsigned long long* trace = ws->cta_trace;
-    ws->last_grid = (int)G;
+    const double z = normal_quantile_upper(1.0 - pq);
+    ws->last_grid = (int)geo.G;
     stage_mark(ws, st, 0);
-    GK_CUDA_TRY(launch_fused(G, st, g, eps, d, k, z, rpc, u_slots, table_rows, ctrl, partials, cta_counts, bars,
-                             idx_out, val_out, nnz_out, cap, trace));
+    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ws->ctrl, ws->partials, ws->cta_counts, ws->bars, ws->rowcnt,
+                             idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_fused = true;
+    ws->phase_spans = 6;
     return GK_OK;
 }
 
@@ -741,9 +643,10 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
 // synchronises the whole device, or a step that has to behave the same on its
 // first and on its millionth call.  For them the scratch of the fused kernel
 // (control block, per-CTA partial sums, per-CTA candidate counts, barrier
-// counters) lives in the fixed array below instead of a workspace obtained
-// from cudaMalloc.  The array is part of the library image: every GPU that
-// loads the library holds these 32 KB until the process exits.
+// counters, one word per row of the vector) lives in the fixed array below
+// instead of a workspace obtained from cudaMalloc.  The array is part of the
+// library image: every GPU that loads the library holds these 544 KB until the
+// process exits.
 // ---------------------------------------------------------------------------
 namespace gk {
 
@@ -751,8 +654,10 @@ constexpr size_t kStaticCtrlBytes = (sizeof(Ctrl) + 255) / 256 * 256;
 constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap;                // 8 KB
 constexpr size_t kStaticCountBytes = sizeof(unsigned int) * kFusedGridCap * kNumCand;  // 20 KB
 constexpr size_t kStaticBarBytes = 256;
-constexpr size_t kStaticScratchBytes = 32 * 1024;
-static_assert(kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes + kStaticBarBytes <= kStaticScratchBytes,
+constexpr size_t kStaticHeadBytes = 32 * 1024;             // everything but the per-row words
+constexpr int kStaticRowCap = 1 << 17;                     // rows of 4096 elements: d up to 2^29
+constexpr size_t kStaticScratchBytes = kStaticHeadBytes + sizeof(unsigned int) * kStaticRowCap;  // 544 KB
+static_assert(kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes + kStaticBarBytes <= kStaticHeadBytes,
               "static scratch too small");
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -804,19 +709,19 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
     unsigned int* bars =
         reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes);
 
-    FusedGeometry geo = fused_geometry(d, plan->grid);
-    int64_t G = geo.G;
-    if (G > kFusedGridCap) return GK_ERR_LIMIT;  // more CTAs than the fixed array has slots for
+    unsigned int* rowcnt = reinterpret_cast<unsigned int*>(ss->base + kStaticHeadBytes);
+
+    const FusedGeometry geo = fused_geometry(d, plan->grid);
+    // more CTAs or rows than the fixed array has slots for, or more rows per CTA than the kernel takes
+    if (geo.G > kFusedGridCap || geo.n_rows > kStaticRowCap || !geo.fits) return GK_ERR_LIMIT;
     // The array keeps what the last call left.  The barrier counters must start at zero; the
     // kernel resets them when it ends, but a call that was cut short would not have.
     GK_CUDA_TRY(cudaMemsetAsync(bars, 0, kStaticBarBytes, st));
-    int rpc = geo.rpc, u_slots = geo.u_slots, table_rows = geo.table_rows;
     const double pq = 1.0 - (double)k / (double)d;
-    double z = normal_quantile_upper(1.0 - pq);
-    int64_t cap = output_capacity(d);
+    const double z = normal_quantile_upper(1.0 - pq);
     unsigned long long* trace = nullptr;  // no trace array in the fixed scratch
-    GK_CUDA_TRY(launch_fused(G, st, g, eps, d, k, z, rpc, u_slots, table_rows, ctrl, partials, cta_counts, bars,
-                             idx_out, val_out, nnz_out, cap, trace));
+    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, cta_counts, bars, rowcnt, idx_out, val_out,
+                             nnz_out, output_capacity(d), trace));
     note_launch();
     return GK_OK;
 }

@@ -49,7 +49,7 @@ int64_t output_capacity(int64_t d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t ctrl, partials, hist, cta_counts, bars, cta_trace, tile_status, seg, total;
+    size_t ctrl, partials, hist, cta_counts, bars, cta_trace, rowcnt, tile_status, seg, total;
 };
 
 static Layout layout_for(int64_t d, int32_t S) {
@@ -59,8 +59,9 @@ static Layout layout_for(int64_t d, int32_t S) {
     L.partials = at;    at = align_up(at + sizeof(double2) * kMaxPartials, 256);
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
     L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
-    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 4, 256);
+    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 16, 256);
     L.cta_trace = at;   at = align_up(at + sizeof(unsigned long long) * kFusedGridCap * 8, 256);
+    L.rowcnt = at;      at = align_up(at + sizeof(unsigned int) * 2 * ((size_t)(d >> 12) + 2), 256);
     L.tile_status = at; at = align_up(at + sizeof(unsigned long long) * (size_t)num_compact_tiles(d), 256);
     L.seg = at;         at = align_up(at + segmented_scratch_bytes(d, S), 256);
     L.total = at;
@@ -98,6 +99,7 @@ int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out
         ws.cta_counts = reinterpret_cast<unsigned int*>(b + L.cta_counts);
         ws.bars = reinterpret_cast<unsigned int*>(b + L.bars);
         ws.cta_trace = reinterpret_cast<unsigned long long*>(b + L.cta_trace);
+        ws.rowcnt = reinterpret_cast<unsigned int*>(b + L.rowcnt);
         ws.tile_status = reinterpret_cast<unsigned long long*>(b + L.tile_status);
         ws.seg_block = b + L.seg;
         GK_CUDA_TRY(cudaDeviceGetAttribute(&ws.sm_count, cudaDevAttrMultiProcessorCount, dev));
@@ -190,12 +192,12 @@ extern "C" int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages
     *n_stages = ws->n_stages;
     for (int i = 0; i < ws->n_stages; ++i)
         GK_CUDA_TRY(cudaEventElapsedTime(&ms_out[i], ws->ev[i], ws->ev[i + 1]));
-    if (ws->last_fused && ws->n_stages == 1) {
-        // one kernel: after its event time, the three phases from the kernel's own timestamps
+    if (ws->phase_spans > 0 && ws->n_stages == 1) {
+        // one kernel: after its event time, the spans between the kernel's own timestamps
         unsigned long long t[8];
         GK_CUDA_TRY(cudaMemcpy(t, ws->ctrl->phase_t, sizeof(t), cudaMemcpyDeviceToHost));
-        for (int i = 0; i < 6; ++i) ms_out[1 + i] = (float)((double)(t[i + 1] - t[i]) * 1e-6);
-        *n_stages = 7;
+        for (int i = 0; i < ws->phase_spans; ++i) ms_out[1 + i] = (float)((double)(t[i + 1] - t[i]) * 1e-6);
+        *n_stages = 1 + ws->phase_spans;
     }
     return GK_OK;
 }

@@ -376,6 +376,7 @@ extern "C" int gk_sparsify_segmented(const float* g, float* eps, int64_t d, cons
                                   seg_offsets, (int)S, (const float*)v.thr_sel));
     stage_mark(ws, st, 3);
     ws->last_fused = false;
+    ws->phase_spans = 0;
     note_launch(3);
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;

@@ -226,6 +226,7 @@ int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d
     note_launch();
     stage_mark(ws, st, 3);
     ws->last_fused = false;
+    ws->phase_spans = 0;
     GK_CUDA_TRY(cudaGetLastError());
     return GK_OK;
 }

@@ -305,6 +305,11 @@ extern "C" int topk_exact(const float* u, int64_t d, int64_t k, int32_t* idx_out
     Workspace* ws = nullptr;
     const int wrc = acquire_workspace(d, 1, (cudaStream_t)stream, &ws);
     if (wrc != GK_OK) return wrc;
+    if (selected_path() == 0) {
+        const int frc = enqueue_topk_fused(ws, u, nullptr, d, k, idx_out, val_out, nullptr, (cudaStream_t)stream);
+        if (frc != 1) return frc;  // 1: the single-kernel form cannot serve this call
+    }
+    ws->phase_spans = 0;
     return enqueue_topk<false>(ws, const_cast<float*>(u), d, k, idx_out, val_out, (cudaStream_t)stream, 0);
 }
 
@@ -320,6 +325,11 @@ extern "C" int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, i
     Workspace* ws = nullptr;
     const int wrc = acquire_workspace(d, 1, st, &ws);
     if (wrc != GK_OK) return wrc;
+    if (selected_path() == 0) {
+        const int frc = enqueue_topk_fused(ws, g, eps, d, k, idx_out, val_out, nnz_out, st);
+        if (frc != 1) return frc;
+    }
+    ws->phase_spans = 0;
     const int64_t n4 = d >> 2;
     int64_t grid = (n4 + 511) / 512;
     if (grid < 1) grid = 1;

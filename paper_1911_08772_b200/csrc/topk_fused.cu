@@ -1,0 +1,588 @@
+// Exact Top_k (Section 1 of arXiv 1911.08772) as ONE persistent cooperative
+// kernel: most-significant-digit radix select on the 31 magnitude bits of the
+// fp32 pattern, followed by the ordered compaction, with what fits of u kept
+// on chip between the passes.
+//
+// The vector is cut into rows of 1024 float4, dealt to one CTA per SM in turn (CTA c owns
+// rows c, c + G, ...), so that every CTA gets the same mix of quiet and loud stretches.
+//
+//   pass 1   the run streams in through asynchronous copies (with ACCUM, g and
+//            eps: u = g + eps goes back over eps, Eq. 2); every key's top 11
+//            bits are counted in a shared-memory histogram; per (row, warp)
+//            segment of 128 elements the largest magnitude goes to a table.
+//   barrier  histograms are merged in global memory; every CTA finds the digit
+//            that holds the k-th largest key.
+//   pass 2/3 the next 10 + 10 bits, among the keys that match the digits found
+//            so far.  Only segments whose recorded maximum reaches the first
+//            digit are read again (a few percent of them when k << d), from
+//            shared memory or L2.
+//   barrier  after the third digit the threshold key T and the number of keys
+//            equal to T still to take are known.
+//   compact  every CTA counts the keys above / equal to T per row (the same few
+//            segments again), the rows' counts are exchanged through a fourth
+//            barrier, which gives every row its output offset -- no look-back;
+//            keys above T are all taken, keys equal to T in order of increasing
+//            index until k pairs are out.
+//
+// All waits are bounded (grid_barrier); a CTA whose wait runs out records
+// GK_DEV_TIMEOUT and leaves.  Vectors whose runs exceed the table (more than
+// kTkTableMaxRows rows per CTA) and devices without cooperative launch take
+// the multi-kernel path in topk_exact.cu.
+#include "gk_common.cuh"
+#include "gk_coop.cuh"
+#include "gk_count.cuh"
+
+namespace gk {
+
+constexpr int kTkTableMaxRows = 448;                                   // rows per CTA the maximum table covers
+constexpr int kTkTableBytes = kTkTableMaxRows * kFusedWarps * 2;       // 28 KB: one uint16 per (row, warp)
+constexpr int kTkSmemRows = 11;                                        // 16 KB rows of dynamic shared memory
+constexpr int kTkSmemBytes = kTkSmemRows * kRowBytes + kTkTableBytes;  // g ring (ACCUM), u slots, table
+constexpr int kTkStages = 4;                                           // rows in flight in pass 1, plus one
+constexpr int kTkGroupRows = 8;                                        // rows a warp gathers per batch
+constexpr int kTkBins = 2048;
+constexpr unsigned short kTkPending = 0xffffu;                         // table entry: segment still to be counted
+
+struct __align__(128) TopkShared {
+    unsigned int hist[kTkBins];      // this CTA's histogram of the current digit
+    unsigned int wsum[kFusedWarps];
+    unsigned long long wsum2[kFusedWarps];
+    // keys above T (low word) and equal to T (high word): per round of G consecutive rows, and
+    // in the vector before each row of this CTA
+    unsigned long long roundtot[kTkTableMaxRows];
+    unsigned long long rowpre[kTkTableMaxRows];
+    unsigned short qrow[kFusedWarps][kTkGroupRows];
+    unsigned long long need;         // entries still to take among the keys that match the digits so far
+    unsigned int digit;
+    int ok;
+};
+static_assert((sizeof(TopkShared) + 1023) / 1024 * 1024 + kTkSmemBytes <= 232448,
+              "over the 227 KB of shared memory per CTA (the dynamic part starts on a 1 KB boundary)");
+
+__device__ __forceinline__ unsigned int tk_key(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+__device__ __forceinline__ unsigned int warp_incl_scan(unsigned int v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_incl_scan64(unsigned long long v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Called by every CTA after a grid barrier.  ghist: the level's NB merged bins.  Finds the
+// largest digit D with  #(keys in bins > D) < need <= #(keys in bins >= D),  leaves D in
+// sh.digit and need - #(keys in bins > D) in sh.need.
+__device__ __forceinline__ void pick_digit(const unsigned int* __restrict__ ghist, int NB, TopkShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const unsigned long long need = sh.need;
+    // thread 0 owns the two highest bins, thread 1 the next two, ...
+    const int hi = NB - 1 - 2 * tid, lo = hi - 1;
+    const unsigned int g_hi = hi >= 0 ? __ldcg(ghist + hi) : 0u;
+    const unsigned int g_lo = lo >= 0 ? __ldcg(ghist + lo) : 0u;
+    const unsigned int mine = g_hi + g_lo;
+    const unsigned int s = warp_incl_scan(mine, lane);
+    if (lane == 31) sh.wsum[w] = s;
+    __syncthreads();
+    const unsigned int x = sh.wsum[lane];
+    const unsigned int y = warp_incl_scan(x, lane);
+    const unsigned int wpre = __shfl_sync(0xffffffffu, y - x, w);
+    const unsigned long long above = (unsigned long long)wpre + s - mine;  // keys in the bins above `hi`
+    __syncthreads();  // every thread has read sh.need and sh.wsum
+    if (above < need && need <= above + mine) {  // true in exactly one thread
+        if (need <= above + g_hi) { sh.digit = (unsigned int)hi; sh.need = need - above; }
+        else { sh.digit = (unsigned int)lo; sh.need = need - above - g_hi; }
+    }
+    __syncthreads();
+}
+
+// Adds this CTA's histogram to the merged one and clears it.
+__device__ __forceinline__ void merge_hist(unsigned int* __restrict__ ghist, int NB, TopkShared& sh) {
+    for (int b = threadIdx.x; b < NB; b += kFusedThreads) {
+        const unsigned int c = sh.hist[b];
+        if (c) { atomicAdd(ghist + b, c); sh.hist[b] = 0u; }
+    }
+}
+
+// ACCUM: src = g, eps in/out (u stored over eps, selected slots cleared).  Otherwise src = u,
+// read-only, eps unused.  n_rows: rows of 1024 float4 in the vector; CTA c owns rows c, c + G,
+// c + 2G, ... so that stretches of large values are spread over all CTAs.  ghist: 2048 + 1024 +
+// 1024 merged bins, zero on entry and on exit.  rowcnt: two words per row of the vector.
+// bars: four barrier counters and an exit counter, zero on entry and on exit.
+// Shared memory: [g ring of kTkStages rows (ACCUM only)][u_slots rows][table].
+template <bool ACCUM>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, int n_rows, int u_slots,
+             Ctrl* __restrict__ ctrl, unsigned int* __restrict__ ghist, uint2* __restrict__ rowcnt,
+             unsigned int* __restrict__ bars, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+             int64_t* __restrict__ nnz_out) {
+    // 1 KB alignment keeps every warp's 512 bytes of a row within four 128-byte lines of shared
+    // memory, whatever the size of the static part
+    extern __shared__ __align__(1024) float4 smem4[];
+    __shared__ TopkShared sh;
+    float4* gring = smem4;
+    float4* uslot = smem4 + (ACCUM ? (size_t)kTkStages * kRowF4 : 0);
+    unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)kTkSmemRows * kRowF4);
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int c = blockIdx.x, G = gridDim.x;
+    const int64_t n4 = d >> 2;
+    unsigned int* ghist1 = ghist;
+    unsigned int* ghist2 = ghist + 2048;
+    unsigned int* ghist3 = ghist + 3072;
+
+    // this CTA's rows: local row r is row c + r * G of the vector (at most kTkTableMaxRows of
+    // them); only the last row of the vector can be short
+    const int nrows = c < n_rows ? (n_rows - c + G - 1) / G : 0;
+    const int64_t stride4 = (int64_t)G * kRowF4;
+    const int64_t first4 = (int64_t)c * kRowF4 + tid;
+    const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on stay on chip
+    const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
+    const int64_t tail_i = (n4 << 2) + lane;
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* e4 = reinterpret_cast<float4*>(eps);
+    const float4* uglob = ACCUM ? reinterpret_cast<const float4*>(eps) : s4;  // where u is after pass 1
+    float tail_u = 0.f;
+    const bool wide_ok = ACCUM && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);
+
+    if (c == 0 && tid == 0) {
+        ctrl->stats.status = GK_DEV_OK;
+        ctrl->phase_t[0] = global_timer_ns();
+        if (nnz_out != nullptr) *nnz_out = k;
+    }
+    for (int b = tid; b < kTkBins; b += kFusedThreads) sh.hist[b] = 0u;
+    if (tid == 0) { sh.need = (unsigned long long)k; sh.digit = 0u; }
+    __syncthreads();
+
+    // up to kTkGroupRows rows of this warp whose table entry is pending (want_pending) or
+    // non-zero, from `cursor` on; they are left in sh.qrow[w]
+    auto gather = [&](int& cursor, const bool want_pending) -> int {
+        int n = 0;
+        while (n < kTkGroupRows && cursor < nrows) {
+            const int r = cursor + lane;
+            unsigned int e = 0u;
+            if (r < nrows) e = table[r * kFusedWarps + w];
+            const bool hit = want_pending ? (e == kTkPending) : (e != 0u);
+            unsigned int b = __ballot_sync(0xffffffffu, hit);
+            while (b && n < kTkGroupRows) {
+                const int bit = __ffs(b) - 1;
+                if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
+                ++n;
+                b &= b - 1u;
+            }
+            if (b) { cursor += __ffs(b) - 1; break; }
+            cursor += 32;
+        }
+        __syncwarp();
+        return n;
+    };
+    // this thread's float4 of local row r (zeros beyond the end of the vector)
+    auto load_row = [&](int r) -> float4 {
+        const int64_t i = first4 + (int64_t)r * stride4;
+        if (i >= n4) return make_float4(0.f, 0.f, 0.f, 0.f);
+        return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(uglob + i);
+    };
+    // body(r, v, in_range) for every marked segment of this warp, rows gathered eight at a time
+    // so that their loads overlap
+#define TK_FOR_EACH_MARKED(want_pending, ...)                                       \
+    for (int cursor_ = 0; cursor_ < nrows;) {                                         \
+        const int n_ = gather(cursor_, want_pending);                                 \
+        float4 v_[kTkGroupRows];                                                      \
+        _Pragma("unroll") for (int q_ = 0; q_ < kTkGroupRows; ++q_) {                 \
+            v_[q_] = make_float4(0.f, 0.f, 0.f, 0.f);                                 \
+            if (q_ < n_) v_[q_] = load_row(sh.qrow[w][q_]);                           \
+        }                                                                             \
+        _Pragma("unroll") for (int q_ = 0; q_ < kTkGroupRows; ++q_) {                 \
+            if (q_ < n_) {                                                            \
+                const int r = sh.qrow[w][q_];                                         \
+                const float4 v = v_[q_];                                              \
+                const bool in = first4 + (int64_t)r * stride4 < n4;                   \
+                __VA_ARGS__                                                           \
+            }                                                                         \
+        }                                                                             \
+        __syncwarp();                                                                 \
+    }
+
+    // ------------------------------------------------------------------ pass 1
+    {
+        int64_t fi = first4;  // the row the next fetch brings in
+        auto fetch = [&](int r) {
+            if (r < nrows && fi < n4) {
+                if (ACCUM) {
+                    cp_async16(gring + (size_t)(r % kTkStages) * kRowF4 + tid, s4 + fi);
+                    cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + fi);
+                } else {
+                    cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, s4 + fi);
+                }
+            }
+            cp_async_commit();
+            fi += stride4;
+        };
+#pragma unroll
+        for (int r = 0; r < kTkStages - 1; ++r) fetch(r);
+        int64_t i = first4;
+        for (int r = 0; r < nrows; ++r, i += stride4) {
+            fetch(r + kTkStages - 1);
+            cp_async_wait<kTkStages - 1>();
+            const bool one = i < n4;
+            float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (one) {
+                float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
+                u0 = *us;
+                if (ACCUM) {
+                    const float4 a0 = gring[(size_t)(r % kTkStages) * kRowF4 + tid];
+                    u0 = make_float4(a0.x + u0.x, a0.y + u0.y, a0.z + u0.z, a0.w + u0.w);
+                    *us = u0;
+                }
+                atomicAdd(&sh.hist[tk_key(u0.x) >> 20], 1u);
+                atomicAdd(&sh.hist[tk_key(u0.y) >> 20], 1u);
+                atomicAdd(&sh.hist[tk_key(u0.z) >> 20], 1u);
+                atomicAdd(&sh.hist[tk_key(u0.w) >> 20], 1u);
+            }
+            if (ACCUM) {
+                // u goes out in 32-byte stores by the even lanes (own float4 and the right
+                // neighbour's), marked to stay in L2: the later passes read parts of u again
+                float4 nb;
+                nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
+                nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
+                const bool pair = wide_ok && (i + 1 < n4);
+                if ((lane & 1) == 0) {
+                    if (pair) st_keep32(e4 + i, u0, nb);
+                    else if (one) e4[i] = u0;
+                } else if (one && !wide_ok) {
+                    e4[i] = u0;
+                }
+            }
+            // largest magnitude of each (row, warp) segment, top 16 bits rounded up
+            const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
+            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
+        }
+        cp_async_wait<0>();
+        if (owns_tail) {
+            tail_u = ACCUM ? src[tail_i] + eps[tail_i] : src[tail_i];
+            if (ACCUM) eps[tail_i] = tail_u;
+            atomicAdd(&sh.hist[tk_key(tail_u) >> 20], 1u);
+        }
+        __syncthreads();
+        merge_hist(ghist1, 2048, sh);
+        if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
+        if (!grid_barrier(&bars[0], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        pick_digit(ghist1, 2048, sh);
+    }
+
+    {
+        const unsigned int b1 = sh.digit;
+        // a segment can hold a key with first digit >= b1 only if its recorded maximum
+        // (top 16 bits, rounded up) reaches b1's lower bound; the others are never read again
+        const unsigned int low16 = b1 << 4;
+        for (int r = lane; r < nrows; r += 32) {
+            const bool ql = table[r * kFusedWarps + w] >= low16;
+            table[r * kFusedWarps + w] = ql ? kTkPending : (unsigned short)0;
+        }
+        if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
+        __syncthreads();
+
+        // -------------------------------------------------------------- pass 2
+        TK_FOR_EACH_MARKED(true, {
+            if (in) {
+                const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    if ((key[t] >> 20) == b1) atomicAdd(&sh.hist[(key[t] >> 10) & 1023u], 1u);
+            }
+        })
+        if (owns_tail && (tk_key(tail_u) >> 20) == b1) atomicAdd(&sh.hist[(tk_key(tail_u) >> 10) & 1023u], 1u);
+        __syncthreads();
+        merge_hist(ghist2, 1024, sh);
+        if (!grid_barrier(&bars[1], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        // every CTA has read the first level's merged bins before it arrived here
+        if (c == 0) for (int b = tid; b < 2048; b += kFusedThreads) ghist1[b] = 0u;
+        pick_digit(ghist2, 1024, sh);
+        const unsigned int p21 = (b1 << 10) | sh.digit;
+        if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
+
+        // -------------------------------------------------------------- pass 3
+        TK_FOR_EACH_MARKED(true, {
+            if (in) {
+                const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    if ((key[t] >> 10) == p21) atomicAdd(&sh.hist[key[t] & 1023u], 1u);
+            }
+        })
+        if (owns_tail && (tk_key(tail_u) >> 10) == p21) atomicAdd(&sh.hist[tk_key(tail_u) & 1023u], 1u);
+        __syncthreads();
+        merge_hist(ghist3, 1024, sh);
+        if (!grid_barrier(&bars[2], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        if (c == 0) for (int b = tid; b < 1024; b += kFusedThreads) ghist2[b] = 0u;
+        pick_digit(ghist3, 1024, sh);
+        const unsigned int T = (p21 << 10) | sh.digit;
+        const unsigned long long need_eq = sh.need;  // >= 1: entries equal to T to take, lowest indices first
+        if (c == 0 && tid == 0) {
+            ctrl->key_threshold = T;
+            ctrl->need_eq = need_eq;
+            ctrl->phase_t[4] = global_timer_ns();
+        }
+
+        // ---------------------------------------------------------- compaction
+        // step 1: every warp counts the keys above / equal to T of its marked segments; the
+        // table entry becomes (above) | (equal << 8), at most 128 each
+        TK_FOR_EACH_MARKED(true, {
+            unsigned int g = 0u, e = 0u;
+            if (in) {
+                const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) { g += key[t] > T; e += key[t] == T; }
+            }
+            const unsigned int ge = __reduce_add_sync(0xffffffffu, g | (e << 8));
+            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)ge;
+        })
+        __syncthreads();
+        // step 2: per row (thread t takes local row t) the two counts go to the row's words in
+        // global memory; every row of the vector gets them from the CTA that owns it
+        bool any_mine = false;
+        if (tid < nrows) {
+            const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
+            unsigned int lo8 = 0u, hi8 = 0u;
+#pragma unroll
+            for (int q = 0; q < kFusedWarps * 2 / 16; ++q) {
+                const uint4 x = tv[q];
+                const unsigned int ws[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    lo8 += (ws[j] & 0xffu) + ((ws[j] >> 16) & 0xffu);
+                    hi8 += ((ws[j] >> 8) & 0xffu) + (ws[j] >> 24);
+                }
+            }
+            rowcnt[c + tid * G] = make_uint2(lo8, hi8);
+            any_mine = (lo8 | hi8) != 0u;
+        }
+        any_mine = __syncthreads_or(any_mine) != 0;
+        if (!grid_barrier(&bars[3], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        if (c == 0) for (int b = tid; b < 1024; b += kFusedThreads) ghist3[b] = 0u;
+        if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
+        const bool tail_cta = (c == G - 1) && (d & 3);
+        unsigned long long all_rows = 0ull;  // keys above / equal to T in all rows (tail CTA only)
+        if (any_mine || tail_cta) {
+            // Keys above / equal to T before local row r of this CTA = those of the rounds before r
+            // (round r is the G consecutive rows r * G ... r * G + G - 1) + those of the CTAs
+            // before this one in round r.  Warp j takes rounds j, j + 32, ...; a count pair
+            // travels as one 64-bit word (above in the low half, equal in the high half).
+            for (int r = w; r < nrows; r += kFusedWarps) {
+                unsigned long long tot = 0ull, pre = 0ull;
+                const int R0 = r * G;
+                for (int t = lane; t < G; t += 32) {
+                    uint2 x = make_uint2(0u, 0u);
+                    if (R0 + t < n_rows) x = __ldcg(rowcnt + R0 + t);
+                    const unsigned long long v = (unsigned long long)x.x | ((unsigned long long)x.y << 32);
+                    tot += v;
+                    pre += (t < c) ? v : 0ull;
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                    pre += __shfl_xor_sync(0xffffffffu, pre, o);
+                }
+                if (lane == 0) { sh.roundtot[r] = tot; sh.rowpre[r] = pre; }
+            }
+            __syncthreads();
+            // exclusive scan of the round totals (thread t takes round t; at most kTkTableMaxRows).
+            // CTA 0 owns a row of every round, so its number of rows is the number of rounds; the
+            // tail CTA may own one row fewer and then adds the last round separately.
+            {
+                const unsigned long long mine_round = tid < nrows ? sh.roundtot[tid] : 0ull;
+                const unsigned long long s = warp_incl_scan64(mine_round, lane);
+                if (lane == 31) sh.wsum2[w] = s;
+                __syncthreads();
+                const unsigned long long x = sh.wsum2[lane];
+                const unsigned long long y = warp_incl_scan64(x, lane);
+                const unsigned long long wpre = __shfl_sync(0xffffffffu, y - x, w);
+                if (tid < nrows) sh.rowpre[tid] += wpre + s - mine_round;
+                all_rows = __shfl_sync(0xffffffffu, y, 31);
+                __syncthreads();
+            }
+        }
+        if (any_mine) {
+            // step 3: every warp writes the selected entries of its segments that have any: keys
+            // above T always, keys equal to T while fewer than need_eq of them came before
+            TK_FOR_EACH_MARKED(false, {
+                unsigned int gm = 0u, em = 0u;
+                if (in) {
+                    const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) { gm |= (unsigned)(key[t] > T) << t; em |= (unsigned)(key[t] == T) << t; }
+                }
+                // counts of this row in the warps before this one, then in the lanes before this one
+                const unsigned int e_before = lane < w ? (unsigned int)table[r * kFusedWarps + lane] : 0u;
+                const unsigned int wb = __reduce_add_sync(0xffffffffu, (e_before & 0xffu) | ((e_before >> 8) << 16));
+                const unsigned int mine_ge = __popc(gm) | (__popc(em) << 16);
+                const unsigned int sc = warp_incl_scan(mine_ge, lane) - mine_ge;
+                if (gm | em) {
+                    const unsigned long long rp = sh.rowpre[r];
+                    unsigned long long ng = (rp & 0xffffffffull) + (wb & 0xffffu) + (sc & 0xffffu);
+                    unsigned long long ne = (rp >> 32) + (wb >> 16) + (sc >> 16);
+                    const int64_t e0 = (first4 + (int64_t)r * stride4) << 2;
+                    const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const bool isg = gm & (1u << t), ise = em & (1u << t);
+                        if (isg || (ise && ne < need_eq)) {
+                            const unsigned long long pos = ng + (ne < need_eq ? ne : need_eq);
+                            if ((long long)pos < k) {
+                                idx_out[pos] = (int32_t)(e0 + t);
+                                val_out[pos] = vv[t];
+                                if (ACCUM) eps[e0 + t] = 0.0f;
+                            }
+                        }
+                        ng += isg; ne += ise;
+                    }
+                }
+            })
+        }
+        // the ragged tail comes last in index order
+        if (tail_cta && w == kFusedWarps - 1) {
+            // rounds this CTA has no row in (the last one, possibly) are missing from its scan
+            unsigned long long extra = 0ull;
+            const int rounds = (n_rows + G - 1) / G;
+            if (rounds > nrows) {
+                for (int t = lane; t < G; t += 32) {
+                    const int R = (rounds - 1) * G + t;
+                    if (R < n_rows) {
+                        const uint2 x = __ldcg(rowcnt + R);
+                        extra += (unsigned long long)x.x | ((unsigned long long)x.y << 32);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) extra += __shfl_xor_sync(0xffffffffu, extra, o);
+            }
+            const unsigned long long tot = all_rows + extra;
+            const unsigned int key = tk_key(tail_u);
+            const bool isg = owns_tail && key > T, ise = owns_tail && key == T;
+            const unsigned int bg = __ballot_sync(0xffffffffu, isg), be = __ballot_sync(0xffffffffu, ise);
+            const unsigned int below = (1u << lane) - 1u;
+            const unsigned long long ng = (tot & 0xffffffffull) + __popc(bg & below);
+            const unsigned long long ne = (tot >> 32) + __popc(be & below);
+            if (isg || (ise && ne < need_eq)) {
+                const unsigned long long pos = ng + (ne < need_eq ? ne : need_eq);
+                if ((long long)pos < k) {
+                    idx_out[pos] = (int32_t)tail_i;
+                    val_out[pos] = tail_u;
+                    if (ACCUM) eps[tail_i] = 0.0f;
+                }
+            }
+        }
+    }
+#undef TK_FOR_EACH_MARKED
+    if (c == 0 && tid == 0) ctrl->phase_t[6] = global_timer_ns();
+
+leave:
+    // the CTA that leaves last clears the barrier counters for the next call
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(&bars[4], 1u);
+        if (t == (unsigned)G - 1) {
+            ctrl->phase_t[7] = global_timer_ns();
+            bars[0] = 0u; bars[1] = 0u; bars[2] = 0u; bars[3] = 0u;
+            __threadfence();
+            bars[4] = 0u;
+        }
+    }
+}
+
+// Host side -----------------------------------------------------------------
+struct TopkPlan {
+    bool ready = false, usable = false;
+    int grid = 0;
+};
+static TopkPlan g_tk_plan[64];
+
+template <bool ACCUM>
+static bool topk_kernel_ready(int sm_count) {
+    if (cudaFuncSetAttribute(k_topk_fused<ACCUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTkSmemBytes) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_topk_fused<ACCUM>, kFusedThreads, kTkSmemBytes) !=
+            cudaSuccess || occ < 1) {
+        cudaGetLastError();
+        return false;
+    }
+    (void)sm_count;
+    return true;
+}
+
+static TopkPlan* topk_plan(int dev, int sm_count) {
+    if (dev < 0 || dev >= 64) return nullptr;
+    TopkPlan& p = g_tk_plan[dev];
+    if (p.ready) return &p;
+    p.ready = true;
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return &p;
+    if (!topk_kernel_ready<false>(sm_count) || !topk_kernel_ready<true>(sm_count)) return &p;
+    p.grid = sm_count < kFusedGridCap ? sm_count : kFusedGridCap;
+    p.usable = true;
+    return &p;
+}
+
+// Returns GK_OK when the fused kernel was enqueued, 1 when it cannot serve this call (the
+// caller then takes the multi-kernel path), or an error.  With eps != nullptr: src = g and
+// u = g + eps is formed, stored over eps and cleared where selected; else src = u, read-only.
+int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                       float* val_out, int64_t* nnz_out, cudaStream_t st) {
+    int dev = 0;
+    GK_CUDA_TRY(cudaGetDevice(&dev));
+    TopkPlan* p = topk_plan(dev, ws->sm_count);
+    if (!p || !p->usable) return 1;
+    const int64_t n4 = d >> 2;
+    const int64_t rows = (n4 + kRowF4 - 1) / kRowF4;
+    int64_t G = rows < p->grid ? rows : p->grid;
+    if (G < 1) G = 1;
+    int64_t most = (rows + G - 1) / G;  // rows of CTA 0
+    if (most < 1) most = 1;
+    if (most > kTkTableMaxRows) return 1;
+    int n_rows = (int)rows;
+    const bool accum = eps != nullptr;
+    int u_slots = accum ? kTkSmemRows - kTkStages : kTkSmemRows;
+    if (u_slots > most) u_slots = (int)most;
+    Ctrl* ctrl = ws->ctrl;
+    unsigned int* ghist = ws->hist;
+    uint2* rowcnt = reinterpret_cast<uint2*>(ws->rowcnt);
+    unsigned int* bars = ws->bars + 4;  // the sparsifier's fused kernel owns the first four counters
+    void* args[] = {(void*)&src, (void*)&eps, (void*)&d, (void*)&k, (void*)&n_rows, (void*)&u_slots, (void*)&ctrl,
+                    (void*)&ghist, (void*)&rowcnt, (void*)&bars, (void*)&idx_out, (void*)&val_out,
+                    (void*)&nnz_out};
+    static_assert(sizeof(args) / sizeof(args[0]) == 13, "k_topk_fused takes 13 arguments");
+    stage_mark(ws, st, 0);
+    const void* fn = accum ? (const void*)k_topk_fused<true> : (const void*)k_topk_fused<false>;
+    GK_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3((unsigned)G), dim3(kFusedThreads), args, (size_t)kTkSmemBytes, st));
+    note_launch();
+    stage_mark(ws, st, 1);
+    ws->last_grid = (int)G;
+    ws->last_fused = false;
+    ws->phase_spans = 7;
+    return GK_OK;
+}
+
+}  // namespace gk

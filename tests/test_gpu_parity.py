@@ -122,15 +122,36 @@ def test_gk_on_a_side_stream(gk_path):
 
 
 # ------------------------------------------------------------------ exact Top_k
-@pytest.mark.parametrize("d", [1, 2, 5, 33, 1025, TILE, TILE + 1, 3 * TILE + 2, 250_001])
-def test_topk_small_sizes(d):
+@pytest.mark.parametrize("d", [1, 2, 3, 4, 5, 33, 1025, 4096, 4099, TILE, TILE + 1, 3 * TILE + 2, 250_001,
+                               1_900_003])
+def test_topk_small_sizes(d, gk_path):
     rng = wl.misc_rng(2000 + d)
     u = rng.standard_normal(d).astype(np.float32)
-    for k in sorted({1, max(1, d // 50), max(1, d // 3), d}):
+    for k in sorted({1, max(1, d // 1000), max(1, d // 50), max(1, d // 3), d}):
         check_topk(u, k)
 
 
-def test_topk_ties_and_zeros():
+def test_topk_ties_across_rows_and_ctas(gk_path):
+    """Heavy ties in a vector of several rows per CTA: the supply of keys equal to the k-th one
+    runs out in the middle of a CTA's run, in its last row, or in the ragged tail."""
+    rng = wl.misc_rng(77)
+    d = 1_300_003
+    u = (np.round(rng.standard_normal(d) * 4) / 4).astype(np.float32)
+    u[1::5] *= -1
+    for k in (1, 17, 1300, 40_000, d // 2, d - 2, d - 1, d):
+        check_topk(u, k)
+    same = np.full(d, 0.75, dtype=np.float32)
+    same[2::7] = -0.75
+    for k in (1, 4096, 4097, 600_000, d - 3, d - 2, d - 1, d):
+        idx, _ = check_topk(same, k)
+        assert idx[0] == 0 and idx[-1] == k - 1
+    # one large entry in the ragged tail, ties everywhere else
+    same[d - 1] = 9.0
+    idx, _ = check_topk(same, 5)
+    assert idx.tolist() == [0, 1, 2, 3, d - 1]
+
+
+def test_topk_ties_and_zeros(gk_path):
     rng = wl.misc_rng(5)
     d = 2 * TILE + 77
     u = (np.round(rng.standard_normal(d) * 2) / 2).astype(np.float32)  # heavy ties, many +-0
@@ -148,11 +169,10 @@ def test_topk_ties_and_zeros():
     check_topk(tiny, 3)
 
 
-def test_topk_sparsify_matches_eq2_with_exact_topk():
-    d = 3 * TILE + 9
+@pytest.mark.parametrize("d,k", [(3 * TILE + 9, 123), (7, 7), (5, 2), (2_000_003, 2001), (2_000_003, 1_000_000)])
+def test_topk_sparsify_matches_eq2_with_exact_topk(d, k, gk_path):
     g = wl.laplace(d, 1.0, step=21)
     e = wl.normal(d, 0.5, step=22)
-    k = 123
     dev = torch.device("cuda:0")
     dg, de = torch.from_numpy(g).to(dev), torch.from_numpy(e).to(dev)
     idx = torch.empty(k, dtype=torch.int32, device=dev)
