@@ -38,7 +38,9 @@ constexpr int kTkTableMaxRows = 448;                                   // rows p
 constexpr int kTkTableBytes = kTkTableMaxRows * kFusedWarps * 2;       // 28 KB: one uint16 per (row, warp)
 constexpr int kTkSmemRows = 11;                                        // 16 KB rows of dynamic shared memory
 constexpr int kTkSmemBytes = kTkSmemRows * kRowBytes + kTkTableBytes;  // g ring (ACCUM), u slots, table
-constexpr int kTkStages = 4;                                           // rows in flight in pass 1, plus one
+// rows in flight in pass 1, plus one: with ACCUM every row is two copies (g and eps), else one,
+// and about 100 KB in flight per SM are what it takes to keep HBM busy
+template <bool ACCUM> struct TkStages { static constexpr int value = ACCUM ? 4 : 8; };
 constexpr int kTkGroupRows = 8;                                        // rows a warp gathers per batch
 constexpr int kTkBins = 2048;
 constexpr unsigned short kTkPending = 0xffffu;                         // table entry: segment still to be counted
@@ -117,7 +119,7 @@ __device__ __forceinline__ void merge_hist(unsigned int* __restrict__ ghist, int
 // c + 2G, ... so that stretches of large values are spread over all CTAs.  ghist: 2048 + 1024 +
 // 1024 merged bins, zero on entry and on exit.  rowcnt: two words per row of the vector.
 // bars: four barrier counters and an exit counter, zero on entry and on exit.
-// Shared memory: [g ring of kTkStages rows (ACCUM only)][u_slots rows][table].
+// Shared memory: [g ring of kStages rows (ACCUM only)][u_slots rows][table].
 template <bool ACCUM>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, int n_rows, int u_slots,
@@ -129,7 +131,8 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
     extern __shared__ __align__(1024) float4 smem4[];
     __shared__ TopkShared sh;
     float4* gring = smem4;
-    float4* uslot = smem4 + (ACCUM ? (size_t)kTkStages * kRowF4 : 0);
+    constexpr int kStages = TkStages<ACCUM>::value;
+    float4* uslot = smem4 + (ACCUM ? (size_t)kStages * kRowF4 : 0);
     unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)kTkSmemRows * kRowF4);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int c = blockIdx.x, G = gridDim.x;
@@ -216,7 +219,7 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         auto fetch = [&](int r) {
             if (r < nrows && fi < n4) {
                 if (ACCUM) {
-                    cp_async16(gring + (size_t)(r % kTkStages) * kRowF4 + tid, s4 + fi);
+                    cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, s4 + fi);
                     cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + fi);
                 } else {
                     cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, s4 + fi);
@@ -226,18 +229,18 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
             fi += stride4;
         };
 #pragma unroll
-        for (int r = 0; r < kTkStages - 1; ++r) fetch(r);
+        for (int r = 0; r < kStages - 1; ++r) fetch(r);
         int64_t i = first4;
         for (int r = 0; r < nrows; ++r, i += stride4) {
-            fetch(r + kTkStages - 1);
-            cp_async_wait<kTkStages - 1>();
+            fetch(r + kStages - 1);
+            cp_async_wait<kStages - 1>();
             const bool one = i < n4;
             float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one) {
                 float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
                 u0 = *us;
                 if (ACCUM) {
-                    const float4 a0 = gring[(size_t)(r % kTkStages) * kRowF4 + tid];
+                    const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid];
                     u0 = make_float4(a0.x + u0.x, a0.y + u0.y, a0.z + u0.z, a0.w + u0.w);
                     *us = u0;
                 }
@@ -555,6 +558,10 @@ int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, i
     GK_CUDA_TRY(cudaGetDevice(&dev));
     TopkPlan* p = topk_plan(dev, ws->sm_count);
     if (!p || !p->usable) return 1;
+    // With more than one selected entry per 128-element segment on average nearly every
+    // segment is read again in every later pass, through gathers; on large vectors the
+    // streaming passes of the multi-kernel form are then faster (measured: from about 2^25).
+    if (k * 128 > d && d > (int64_t(1) << 25)) return 1;
     const int64_t n4 = d >> 2;
     const int64_t rows = (n4 + kRowF4 - 1) / kRowF4;
     int64_t G = rows < p->grid ? rows : p->grid;
@@ -564,7 +571,10 @@ int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, i
     if (most > kTkTableMaxRows) return 1;
     int n_rows = (int)rows;
     const bool accum = eps != nullptr;
-    int u_slots = accum ? kTkSmemRows - kTkStages : kTkSmemRows;
+    // a slot is reused kStages - 1 rows later at the earliest: u_slots >= kStages in both forms
+    int u_slots = accum ? kTkSmemRows - TkStages<true>::value : kTkSmemRows;
+    static_assert(kTkSmemRows - TkStages<true>::value >= TkStages<true>::value && kTkSmemRows >= TkStages<false>::value,
+                  "not enough row slots for the rows in flight");
     if (u_slots > most) u_slots = (int)most;
     Ctrl* ctrl = ws->ctrl;
     unsigned int* ghist = ws->hist;
