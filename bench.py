@@ -373,6 +373,22 @@ def run_ours(args):
     ms_topk, ms_topk_sp = topk["fused"]["topk_exact_ms"], topk["fused"]["topk_sparsify_ms"]
     del eps2, us
 
+    # ---- the error ratio of Eq. 5 for one Gaussian_k step and one Top_k step from eps = 0
+    diag = {"bound_eq4_1_minus_k_over_d": 1.0 - k / d, "bound_theorem1_squared": (1.0 - k / d) ** 2}
+    eps3 = torch.zeros_like(epss[0])
+    for name, fn in (("gaussiank", gk.gk_sparsify), ("topk", gk.topk_sparsify)):
+        eps3.zero_()
+        fn(gs[0], eps3, k, idx, val, nnz)
+        gk.gk_stage_timing(True)
+        acc = 0.0
+        for _ in range(10):
+            r = gk.gk_error_ratio(eps3, val, nnz)
+            acc += gk.gk_last_stage_ms()[0]
+        gk.gk_stage_timing(False)
+        diag[name] = {"error_ratio": r[0], "nnz": int(nnz.item()), "ms": acc / 10,
+                      "gbs_4B_per_elem": 4.0 * d / (acc / 10) / 1e6}
+    del eps3
+
     # ---- end to end through the host-buffer entry point (pinned host memory)
     hg = [torch.from_numpy(w.grad(j, None)).pin_memory() for j in range(2)]
     heps = torch.zeros(d, dtype=torch.float32).pin_memory()
@@ -424,7 +440,7 @@ def run_ours(args):
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
                  "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
-        "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
+        "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
         "clocks": sampler.summary(),
     }
     print(json.dumps(line))

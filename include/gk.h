@@ -150,6 +150,23 @@ int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k, int32_t* 
                      float* val_out, int64_t* nnz_out, gk_stats* stats_out);
 
 /*
+ * gk_error_ratio -- the compression error ratio of Eq. 5 / Section 3.2 of the
+ * paper, ||u - Comp(u)||^2 / ||u||^2, for a step that has just run (any of the
+ * sparsifiers above): eps then holds u - Comp(u) with the selected slots at
+ * zero, so ||u||^2 = ||eps||^2 + ||val||^2.  Hold it against 1 - k/d (Eq. 4)
+ * and (1 - k/d)^2 (Theorem 1).
+ *
+ *   eps      DEVICE in   d floats: the residual the step left (16-byte aligned)
+ *   val      DEVICE in   the selected values the step wrote
+ *   nnz      DEVICE in   one int64: how many of them
+ *   host_out HOST   out  3 doubles: the ratio, ||u - Comp(u)||^2, ||u||^2
+ * One pass over eps in fp64, deterministic.  Enqueued on `stream`, which is then
+ * synchronised.  A zero vector gives ratio 0.
+ */
+int gk_error_ratio(const float* eps, int64_t d, const float* val, const int64_t* nnz,
+                   gk_stream_t stream, double* host_out);
+
+/*
  * gk_sparsify_static -- gk_sparsify for callers that must not allocate device
  * memory (the paper has no counterpart: this is a deployment variant of the
  * same step, not another method).  Think of a step that runs under a framework

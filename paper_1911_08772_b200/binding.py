@@ -23,6 +23,7 @@ EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
+    "gk_error_ratio",
 ]
 
 
@@ -73,6 +74,8 @@ def load() -> C.CDLL:
     L.gk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     L.gk_sparsify_static.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     L.gk_sparsify_static.restype = C.c_int
+    L.gk_error_ratio.argtypes = [vp, i64, vp, vp, vp, C.POINTER(C.c_double)]
+    L.gk_error_ratio.restype = C.c_int
     L.gk_sparsify_segmented.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.topk_exact.argtypes = [vp, i64, i64, vp, vp, vp]
     L.topk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
@@ -144,6 +147,16 @@ def gk_sparsify_static(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
     _check(load().gk_sparsify_static(_dev(g, torch.float32), _dev(eps, torch.float32), d, k,
                                      _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
                                      _dev(nnz_out, torch.int64), _stream()))
+
+
+def gk_error_ratio(eps, val, nnz):
+    """(ratio, ||u - Comp(u)||^2, ||u||^2) of the step that left `eps` as its residual and wrote
+    the values `val[:nnz]` (Eq. 5 of the paper).  Synchronises the stream."""
+    import torch
+    out = (C.c_double * 3)()
+    _check(load().gk_error_ratio(_dev(eps, torch.float32), eps.numel(), _dev(val, torch.float32),
+                                 _dev(nnz, torch.int64), _stream(), out))
+    return float(out[0]), float(out[1]), float(out[2])
 
 
 def gk_sparsify_segmented(g, eps, seg_offsets, seg_k, idx_out, val_out, seg_nnz_out, nnz_out) -> None:

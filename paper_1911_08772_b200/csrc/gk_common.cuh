@@ -61,6 +61,8 @@ struct Ctrl {
     // thresholds, after its counting loop, after the second barrier, after the replay of the
     // rounds, at the end of its compaction; and of the CTA that leaves last
     unsigned long long phase_t[8];
+    // gk_error_ratio: ratio, ||u - Comp(u)||^2, ||u||^2
+    double diag[4];
 };
 
 struct Workspace {

@@ -187,6 +187,41 @@ def test_topk_sparsify_matches_eq2_with_exact_topk(d, k, gk_path):
     assert np.array_equal(bits(de.cpu().numpy()), bits(orc.residual(u, oi, ov)))
 
 
+# ------------------------------------------------------------------ error ratio (Eq. 5)
+@pytest.mark.parametrize("d,k", [(1, 1), (6, 2), (4099, 40), (250_001, 250), (2_000_003, 20_000)])
+def test_error_ratio_after_gaussiank_and_topk(d, k):
+    """||u - Comp(u)||^2 / ||u||^2 from the residual and the values sent, against the oracle's
+    Eq. 5 evaluated on u and the kept positions, for Gaussian_k and for exact Top_k."""
+    g = wl.normal(d, 1.0, step=31)
+    e = wl.laplace(d, 0.3, step=32)
+    u = orc.accumulate(g, e)
+    dev = torch.device("cuda:0")
+    for which in ("gaussiank", "topk"):
+        dg, de = torch.from_numpy(g).to(dev), torch.from_numpy(e).to(dev)
+        idx = torch.empty(d, dtype=torch.int32, device=dev)
+        val = torch.empty(d, dtype=torch.float32, device=dev)
+        nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+        if which == "gaussiank":
+            gk.gk_sparsify(dg, de, k, idx, val, nnz)
+        else:
+            gk.topk_sparsify(dg, de, k, idx, val, nnz)
+        ratio, err2, all2 = gk.gk_error_ratio(de, val, nnz)
+        n = int(nnz.item())
+        kept = idx[:n].cpu().numpy()
+        expect = orc.error_ratio(u, kept)
+        assert abs(ratio - expect) <= 1e-10, (which, ratio, expect)
+        u64 = u.astype(np.float64)
+        assert abs(all2 - float(np.dot(u64, u64))) <= 1e-10 * all2
+        assert abs(err2 - ratio * all2) <= 1e-10 * all2
+        if which == "topk":
+            assert ratio <= (1.0 - k / d) + 1e-12           # Eq. 4 holds for every u
+    # a zero vector: nothing to lose
+    z = torch.zeros(4099, device=dev)
+    val = torch.zeros(8, device=dev)
+    nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+    assert gk.gk_error_ratio(z, val, nnz) == (0.0, 0.0, 0.0)
+
+
 # ------------------------------------------------------------------ segmented
 def _dev_i64(a):
     return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int64)).to("cuda:0")

@@ -68,6 +68,12 @@ def test_argument_validation_happens_on_the_host(lib):
     assert lib.gk_sparsify_segmented(a, a + 4096, 10, a, a, 0, a, a, None, a, st) == -2
     assert lib.gk_sparsify_segmented(a, a + 4096, 10, a, a, 70000, a, a, None, a, st) == -2
     assert lib.topk_sparsify(a, a + 16, 10, 1, a, a, a, st) == -5
+    import ctypes
+    out = (ctypes.c_double * 3)()
+    assert lib.gk_error_ratio(None, 10, a, a, st, out) == -1
+    assert lib.gk_error_ratio(a, 10, a, a, st, None) == -1
+    assert lib.gk_error_ratio(a, 0, a, a, st, out) == -2
+    assert lib.gk_error_ratio(a + 4, 10, a, a, st, out) == -4
     assert lib.gk_set_capacity(-1) == -8
     assert lib.gk_set_capacity(0) == 0
 
