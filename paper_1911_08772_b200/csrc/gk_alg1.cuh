@@ -89,28 +89,46 @@ __device__ inline void alg1_thresholds(const Alg1State& a, double s1, double s2,
     *a.thr_sel = __double2float_rd(st.thres0);
 }
 
-// Replay of the loop of Algorithm 1 on the candidate counts.  One thread.
-// Returns the index of the candidate whose mask is returned (-1: everything).
-__device__ inline int alg1_resolve(const Alg1State& a, int64_t k) {
-    gk_stats st = *a.stats;
-    if (st.rounds == 0 && st.thr_final == -INFINITY) return -1;  // everything selected
-    int h = 0, b = 0, chosen = 0;
+// Replay of the loop of Algorithm 1 on the ten candidate counts: which candidates the rounds
+// visit, what each of them counts, and which one's mask is returned (the last one evaluated).
+struct Alg1Path {
+    int chosen;                  // candidate index of the returned mask
+    int rounds;                  // rounds executed
+    long long est[kMaxRounds];   // the count seen in each round
+};
+__device__ inline Alg1Path alg1_replay(const unsigned long long* counts, int64_t k) {
+    Alg1Path p;
+    p.chosen = 0;
+    p.rounds = 0;
+    for (int r = 0; r < kMaxRounds; ++r) p.est[r] = 0;
+    int h = 0, b = 0;
     for (int r = 0; r < kMaxRounds; ++r) {
         const int ci = cand_index(h, b);
         // the counts may live in global or in shared memory: a generic volatile load serves both
-        const long long est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&a.counts[ci]);
-        st.counts[r] = est;
-        st.rounds = r + 1;
-        st.thr_final = a.cand64[ci];  // the mask of this round is the last one evaluated
-        st.nnz = est;
-        *a.thr_sel = a.cand32[ci];
-        chosen = ci;
+        const long long est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&counts[ci]);
+        p.est[r] = est;
+        p.rounds = r + 1;
+        p.chosen = ci;
         if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
         else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
         else break;
     }
+    return p;
+}
+
+// The same with the record filled in.  One thread.
+// Returns the index of the candidate whose mask is returned (-1: everything).
+__device__ inline int alg1_resolve(const Alg1State& a, int64_t k) {
+    gk_stats st = *a.stats;
+    if (st.rounds == 0 && st.thr_final == -INFINITY) return -1;  // everything selected
+    const Alg1Path p = alg1_replay(a.counts, k);
+    for (int r = 0; r < p.rounds; ++r) st.counts[r] = p.est[r];
+    st.rounds = p.rounds;
+    st.thr_final = a.cand64[p.chosen];  // the mask of the last round evaluated
+    st.nnz = p.est[p.rounds - 1];
+    *a.thr_sel = a.cand32[p.chosen];
     *a.stats = st;
-    return chosen;
+    return p.chosen;
 }
 #endif
 

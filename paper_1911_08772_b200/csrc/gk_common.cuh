@@ -75,7 +75,7 @@ struct Workspace {
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
     unsigned int* cta_counts = nullptr;     // fused kernel: kFusedGridCap x kNumCand
-    unsigned int* bars = nullptr;           // 16 counters: [0..2] barriers and exit of the fused sparsifier, [4..8] of the fused Top_k
+    unsigned int* bars = nullptr;           // 16 counters: [0..3] fused sparsifier, [4..8] fused Top_k, [10..13] fused segmented
     unsigned int* rowcnt = nullptr;         // fused kernels: two words per row of 4096 elements
     unsigned long long* cta_trace = nullptr;  // fused kernel: kFusedGridCap x 8 timestamps (tracing aid)
     int last_grid = 0;                      // CTAs of the last fused launch
@@ -101,6 +101,9 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
                      float* val_out, int64_t* nnz_out, cudaStream_t st);
 int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                        float* val_out, int64_t* nnz_out, cudaStream_t st);
+int enqueue_gk_fused_seg(Workspace* ws, const float* g, float* eps, int64_t d, const int64_t* seg_offsets,
+                         const int64_t* seg_k, int32_t S, int32_t* idx_out, float* val_out, int64_t* seg_nnz_out,
+                         int64_t* nnz_out, cudaStream_t st);
 int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                         float* val_out, int64_t* nnz_out, cudaStream_t st);
 

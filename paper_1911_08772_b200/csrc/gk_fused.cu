@@ -589,7 +589,9 @@ static FusedGeometry fused_geometry(int64_t d, int grid) {
     const int64_t left = (int64_t)kFusedSmemBudget - (int64_t)kRing * kRowBytes - (int64_t)q.table_rows * kTableRowBytes;
     q.u_slots = (int)(left / kRowBytes);
     if (q.u_slots > most) q.u_slots = (int)most;
-    if (q.u_slots < 1) q.fits = false;
+    // a slot is written again kStages - 1 rows later: with fewer slots than rows in flight the
+    // copy for a later row would land on the row being read
+    if (q.u_slots < kStages && q.u_slots < most) q.fits = false;
     q.smem = (size_t)(kRing + q.u_slots) * kRowBytes + (size_t)q.table_rows * kTableRowBytes;
     return q;
 }

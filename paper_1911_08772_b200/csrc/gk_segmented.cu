@@ -353,6 +353,11 @@ extern "C" int gk_sparsify_segmented(const float* g, float* eps, int64_t d, cons
     Workspace* ws = nullptr;
     const int wrc = acquire_workspace(d, S, st, &ws);
     if (wrc != GK_OK) return wrc;
+    if (selected_path() == 0) {
+        const int frc = enqueue_gk_fused_seg(ws, g, eps, d, seg_offsets, seg_k, S, idx_out, val_out, seg_nnz_out,
+                                             nnz_out, st);
+        if (frc != 1) return frc;  // 1: the single-kernel form cannot serve this call
+    }
     const SegScratch v = segmented_views(ws);
     const int n_tiles = (int)num_compact_tiles(d);
     // contiguous float4 runs of r4 per CTA, no CTA empty

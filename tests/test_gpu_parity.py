@@ -227,7 +227,7 @@ def _dev_i64(a):
     return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int64)).to("cuda:0")
 
 
-def test_segmented_small_and_ragged():
+def test_segmented_small_and_ragged(gk_path):
     offsets = np.array([0, 1, 1, 3, 10, 64, 65, 1000, 1003, 5000, 5000, 9001, 3 * TILE + 6, 4 * TILE + 1],
                        dtype=np.int64)
     d = int(offsets[-1])
@@ -243,7 +243,7 @@ def test_segmented_small_and_ragged():
         check_segmented_step(step, g, e, offsets, seg_k, _dev_i64(offsets), _dev_i64(seg_k), nn)
 
 
-def test_segmented_single_segment_equals_whole_vector():
+def test_segmented_single_segment_equals_whole_vector(gk_path):
     d = 2 * TILE + 11
     g = wl.normal(d, 1e-2, step=5)
     z = np.zeros(d, np.float32)
@@ -257,7 +257,30 @@ def test_segmented_single_segment_equals_whole_vector():
     assert sts[0].thr_final == st.thr_final or abs(sts[0].thr_final / st.thr_final - 1) < 1e-12
 
 
-def test_segmented_bad_table_is_reported_not_fatal():
+@pytest.mark.parametrize("S,d", [(256, 700_003), (257, 700_003), (200, 5_000), (40, 3_000_001)])
+def test_segmented_many_segments_across_rows_and_ctas(S, d, gk_path):
+    """Random tables: boundaries inside rows and inside float4 groups, empty segments, segments
+    that select everything, runs of several CTAs in one segment and many segments in one row;
+    256 segments is the most the single-kernel form takes, 257 goes to the three-kernel form."""
+    rng = wl.misc_rng(900 + S)
+    cuts = np.sort(rng.integers(0, d + 1, size=S - 1))
+    cuts[: S // 10] = np.sort(rng.integers(0, min(d, 6000) + 1, size=S // 10))   # a crowd at the start
+    cuts = np.sort(cuts)
+    offsets = np.concatenate([[0], cuts, [d]]).astype(np.int64)
+    offsets[5] = offsets[4]          # an empty segment
+    sizes = np.diff(offsets)
+    scale = np.repeat(rng.uniform(1e-4, 1e-1, S), sizes)
+    g = (rng.standard_normal(d) * scale).astype(np.float32)
+    e = (rng.standard_normal(d) * scale * 0.5).astype(np.float32)
+    seg_k = np.array([max(1, wl.ceil_k(int(n), 1, 50)) for n in sizes], dtype=np.int64)
+    seg_k[::7] = 10 ** 9             # more than the segment holds: everything is selected there
+    step = DeviceStep(d)
+    nn = torch.zeros(S, dtype=torch.int64, device="cuda:0")
+    eps, _ = check_segmented_step(step, g, e, offsets, seg_k, _dev_i64(offsets), _dev_i64(seg_k), nn)
+    check_segmented_step(step, g, eps, offsets, seg_k, _dev_i64(offsets), _dev_i64(seg_k), nn)
+
+
+def test_segmented_bad_table_is_reported_not_fatal(gk_path):
     d = 20_000
     g = wl.normal(d, 1e-2, step=6)
     offsets = np.array([0, 9000, 8000, d], dtype=np.int64)  # not ascending
@@ -304,7 +327,17 @@ def test_workload_vgg16_laplace_mixture_100_steps():
 def test_workload_resnet50_three_kernel_path():
     gk.gk_set_path(1)
     try:
-        _ec_loop(wl.resnet50_segmented(), "1e-3", 5)
+        w = wl.resnet50_segmented()
+        _ec_loop(w, "1e-3", 5)
+        # and the layer-wise call in its three-kernel form
+        part = w.partition
+        seg_k = part.seg_k(*wl.RHO["1e-3"])
+        step = DeviceStep(w.d)
+        dev_off, dev_k = _dev_i64(part.offsets), _dev_i64(seg_k)
+        nn = torch.zeros(part.S, dtype=torch.int64, device="cuda:0")
+        eps = np.zeros(w.d, dtype=np.float32)
+        for t in range(3):
+            eps, _ = check_segmented_step(step, w.grad(t, None), eps, part.offsets, seg_k, dev_off, dev_k, nn)
     finally:
         gk.gk_set_path(0)
 
