@@ -34,6 +34,21 @@ __host__ __device__ inline double normal_quantile_upper(double q) {
     return flip ? -z : z;
 }
 
+// The candidates thres0 * 0.5^a * 1.5^b listed by ascending factor: 1/8, 1/4, 3/8, 1/2, 3/4, 1,
+// 9/8, 3/2, 9/4, 27/8.  For thres0 >= 0 this is the ascending order of the thresholds, for
+// thres0 < 0 the descending one (the factors differ by 12 % or more, the roundings of the
+// products by 1e-16, and rounding to fp32 is monotone): no sorting is needed.
+__host__ __device__ constexpr int cand_by_factor(int j) {
+    return j == 0 ? cand_index(3, 0) : j == 1 ? cand_index(2, 0) : j == 2 ? cand_index(2, 1)
+         : j == 3 ? cand_index(1, 0) : j == 4 ? cand_index(1, 1) : j == 5 ? cand_index(0, 0)
+         : j == 6 ? cand_index(1, 2) : j == 7 ? cand_index(0, 1) : j == 8 ? cand_index(0, 2)
+         : cand_index(0, 3);
+}
+// Index of the j-th smallest candidate threshold.
+__host__ __device__ constexpr int cand_ascending(int j, bool thres0_negative) {
+    return cand_by_factor(thres0_negative ? kNumCand - 1 - j : j);
+}
+
 // Where one run of Algorithm 1 keeps its scalars.
 struct Alg1State {
     gk_stats* stats;

@@ -203,12 +203,10 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
             alg1_thresholds(st, tot.x, tot.y, pv, d, k, z);
-            // candidate indices in ascending order of threshold (insertion sort, ten entries)
-            for (int j = 0; j < kNumCand; ++j) {
-                int p = j;
-                while (p > 0 && sh.cand32[sh.order[p - 1]] > sh.cand32[j]) { sh.order[p] = sh.order[p - 1]; --p; }
-                sh.order[p] = j;
-            }
+            // candidate indices in ascending order of threshold
+            const bool neg = sh.stats.thres0 < 0.0;
+#pragma unroll
+            for (int j = 0; j < kNumCand; ++j) sh.order[j] = cand_ascending(j, neg);
         }
         if (tid < kNumCand) sh.cta_counts[tid] = 0u;
         if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();

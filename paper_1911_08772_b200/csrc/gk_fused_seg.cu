@@ -19,8 +19,8 @@
 //   barrier  every CTA replays the rounds for every segment: all thresholds are
 //            known everywhere.
 //   phase C  survivors per (row, warp) with the threshold of each element's
-//            segment; per-row counts exchanged through a third barrier give
-//            every row its output offset; pairs written, slots cleared.
+//            segment; the runs' totals exchanged through a third barrier give
+//            every run its output offset; pairs written, slots cleared.
 //
 // Larger tables, vectors of more than kTableMaxRows rows per SM and devices
 // without cooperative launch take the three-kernel form in gk_segmented.cu.
@@ -61,11 +61,6 @@ struct __align__(128) SegFusedShared {
 };
 constexpr int kSfSmemBudget = (232448 - (int)((sizeof(SegFusedShared) + 1023) / 1024 * 1024));
 
-__device__ __forceinline__ Alg1State seg_state_of(const SegScratch& v, int s) {
-    return Alg1State{&v.stats[s], v.cand64 + (size_t)s * kNumCand, v.cand32 + (size_t)s * kNumCand,
-                     v.counts + (size_t)s * kNumCand, &v.thr_sel[s]};
-}
-
 // First segment s >= from with off[s + 1] > e (the segment that holds element e, skipping
 // empty ones); S when there is none.  Sequential: runs meet few segments.
 __device__ __forceinline__ int seg_advance(const long long* off, int S, int from, int64_t e) {
@@ -89,9 +84,9 @@ __device__ __forceinline__ int seg_find(const long long* off, int S, int64_t e) 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, const int64_t* __restrict__ off_g,
                const int64_t* __restrict__ seg_k, int S, int rows_per_cta, int u_slots, Ctrl* __restrict__ ctrl,
-               SegScratch v, unsigned int* __restrict__ bars, unsigned int* __restrict__ rowcnt,
+               SegScratch v, unsigned int* __restrict__ bars, unsigned int* __restrict__ cta_tot,
                int32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t* __restrict__ seg_nnz_out,
-               int64_t* __restrict__ nnz_out, int64_t cap) {
+               int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
     extern __shared__ __align__(1024) float4 smem4[];
     __shared__ SegFusedShared sh;
     float4* gring = smem4;
@@ -120,6 +115,12 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         ctrl->stats.status = GK_DEV_OK;
         ctrl->phase_t[0] = global_timer_ns();
     }
+    // optional per-CTA trace: start, table read, end of phase A, after barrier 1, thresholds
+    // formed, end of phase B, after barrier 2, end
+    auto stamp = [&](int slot) {
+        if (trace != nullptr && tid == 0) trace[(size_t)c * 8 + slot] = global_timer_ns();
+    };
+    stamp(0);
 
     // rows are fetched kSfStages - 1 ahead by asynchronous copies: g into a ring, eps into the slot
     // that will hold u; the first ones go out before the table is read
@@ -137,41 +138,30 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
     // ------------------------------------------------------------ the table
     // Offsets and pivots go to shared memory; every CTA checks the table for itself.
     int bad = 0;
-    for (int q = tid; q <= S; q += kFusedThreads) sh.off[q] = off_g[q];
+    long long kq = 1;
+    if (tid <= S) sh.off[tid] = off_g[tid];  // S <= kSegFusedMax < the number of threads
+    if (tid < S) kq = seg_k[tid];
     __syncthreads();
     if (tid == 0 && (sh.off[0] != 0 || sh.off[S] != d)) bad = 1;
-    for (int q = tid; q < S; q += kFusedThreads) {
-        const long long a = sh.off[q], b = sh.off[q + 1];
-        if (a < 0 || b > d || b < a || seg_k[q] < 1) bad = 1;
+    if (tid < S) {
+        const long long a = sh.off[tid], b = sh.off[tid + 1];
+        if (a < 0 || b > d || b < a || kq < 1) bad = 1;
     }
     bad = __syncthreads_or(bad);
-    for (int q = tid; q < S; q += kFusedThreads) {
-        const long long a = sh.off[q];
-        sh.piv[q] = (!bad && a < d) ? (double)g[a] : 0.0;
-    }
-    // the normal quantiles depend only on (k_s, d_s): thread t of CTA c takes segment c + t * G
-    {
-        const int64_t q = (int64_t)c + (int64_t)tid * G;
-        if (q < S && !bad) {
-            const long long n = sh.off[q + 1] - sh.off[q];
-            long long kk = seg_k[q];
-            if (kk > n) kk = n;
-            double zq = -INFINITY;
-            if (n > 0 && kk >= 1 && kk < n) {
-                const double pq = 1.0 - (double)kk / (double)n;  // Algorithm 1: p = 1 - k/d
-                zq = normal_quantile_upper(1.0 - pq);
-            }
-            v.zs[q] = zq;
-        }
+    if (tid < S) {
+        const long long a = sh.off[tid];
+        sh.piv[tid] = (!bad && a < d) ? (double)g[a] : 0.0;
     }
     // candidate counts start at zero
     if (c == 0) for (int j = tid; j < S * kNumCand; j += kFusedThreads) v.counts[j] = 0ull;
     __syncthreads();
     const int S_use = bad ? 0 : S;  // a malformed table: u is still formed, nothing is selected
+    stamp(1);
 
     // ------------------------------------------------------------------ phase A
     {
         double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
+        bool dirty = false;                          // this thread has added something for segment s
         int s = seg_find(sh.off, S_use, run_lo);     // the segment the run is in (S_use: none)
         long long send = s < S_use ? sh.off[s + 1] : (long long)d + 1;
         double pv = s < S_use ? sh.piv[s] : 0.0;
@@ -183,13 +173,16 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         auto leave_segment = [&](int64_t e) {
             const int li = s - s_first;
             if (li < kSfLocal) {
-                const double a = warp_sum(s0 + s1), b = warp_sum(q0 + q1);
+                // a short segment lies in a few warps only: the others have nothing to add up
+                double a = 0.0, b = 0.0;
+                if (__any_sync(0xffffffffu, dirty)) { a = warp_sum(s0 + s1); b = warp_sum(q0 + q1); }
                 if (lane == 0) sh.wpart[li][w] = make_double2(a, b);
             } else {
                 const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
                 if (tid == 0) v.partials[c + s] = part;
             }
             s0 = q0 = s1 = q1 = 0.0;
+            dirty = false;
             s = seg_advance(sh.off, S_use, s + 1, e);
             send = s < S_use ? sh.off[s + 1] : (long long)d + 1;
             pv = s < S_use ? sh.piv[s] : 0.0;
@@ -239,6 +232,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                                  x3 = (double)u0.w - pv;
                     s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
                     s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
+                    dirty = true;
                 }
             }
             if (r >= nrows) break;
@@ -256,16 +250,18 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 if (re1 > rows_hi) re1 = rows_hi;
                 const int64_t e0 = (lo4 + (int64_t)r * kRowF4 + tid) << 2;
                 const float uu[4] = {u0.x, u0.y, u0.z, u0.w};
+                const int64_t we0 = re0 + 128 * w;  // this warp's 128 elements of the row
                 int64_t cur = re0;
                 while (cur < re1 && s < S_use) {
                     const int64_t seg_hi = send < re1 ? send : re1;
-                    if (one) {
+                    if (one && we0 < seg_hi && we0 + 128 > cur) {
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
                             const int64_t e = e0 + t;
                             if (e >= cur && e < seg_hi) {
                                 const double x = (double)uu[t] - pv;
                                 s0 += x; q0 = fma(x, x, q0);
+                                dirty = true;
                             }
                         }
                     }
@@ -290,6 +286,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 if (owns_tail && tail_i >= cur && tail_i < seg_hi) {
                     const double x = (double)tail_u - pv;
                     s0 += x; q0 = fma(x, x, q0);
+                    dirty = true;
                 }
                 cur = seg_hi;
                 if (send <= d) leave_segment(cur); else break;
@@ -309,10 +306,30 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 v.partials[c + q] = make_double2(a, b);
             }
         }
+        // The normal quantiles depend only on (k_s, d_s).  Whoever has finished its rows takes
+        // segments from a shared ticket until none is left: the CTAs that are early at the barrier
+        // anyway do most of them.
+        if (tid == 0 && !bad) {
+            while (true) {
+                const unsigned int q = atomicAdd(&bars[4], 1u);
+                if (q >= (unsigned)S) break;
+                const long long n = sh.off[q + 1] - sh.off[q];
+                long long kk = seg_k[q];
+                if (kk > n) kk = n;
+                double zq = -INFINITY;
+                if (n > 0 && kk >= 1 && kk < n) {
+                    const double pq = 1.0 - (double)kk / (double)n;  // Algorithm 1: p = 1 - k/d
+                    zq = normal_quantile_upper(1.0 - pq);
+                }
+                v.zs[q] = zq;
+            }
+        }
+        stamp(2);
         if (!grid_barrier(&bars[0], (unsigned)G, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
+        stamp(3);
     }
 
     // --------------------------------------------------- thresholds of every segment
@@ -326,6 +343,8 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         float c32[kNumCand];
         unsigned long long dummy[kNumCand];
         float tsel;
+#pragma unroll
+        for (int i = 0; i < kNumCand; ++i) { c32[i] = INFINITY; c64[i] = INFINITY; }
         const Alg1State st{&rec, c64, c32, dummy, &tsel};
         bool counted = false;
         if (bad || n <= 0) {
@@ -355,14 +374,14 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         }
         sh.counted[q] = counted ? 1 : 0;
         sh.thr[q] = tsel;
-        // insertion sort of the ten thresholds
-        int od[kNumCand];
+        // the ten thresholds in ascending order (all equal when nothing is counted)
+        const bool neg = counted && rec.thres0 < 0.0;
+#pragma unroll
         for (int j = 0; j < kNumCand; ++j) {
-            int pos = j;
-            while (pos > 0 && c32[od[pos - 1]] > c32[j]) { od[pos] = od[pos - 1]; --pos; }
-            od[pos] = j;
+            const int oj = cand_ascending(j, neg);
+            sh.cs[q][j] = c32[oj];
+            sh.ord[q][j] = (unsigned char)oj;
         }
-        for (int j = 0; j < kNumCand; ++j) { sh.cs[q][j] = c32[od[j]]; sh.ord[q][j] = (unsigned char)od[j]; }
         if (c == 0) {
             v.stats[q] = rec;
             v.thr_sel[q] = tsel;
@@ -375,12 +394,13 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
     for (int j = tid; j < kSfLocal * kNumCand; j += kFusedThreads) (&sh.cnt2[0][0])[j] = 0u;
     if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
     __syncthreads();
+    stamp(4);
 
     // ------------------------------------------------------------------ phase B
     {
         float cs[kNumCand], acc[kNumCand];
         Tiers tier;
-        bool any_neg = false, counted = false;
+        bool any_neg = false, counted = false, dirty = false;
         int s = seg_find(sh.off, S_use, run_lo);
         long long send = s < S_use ? sh.off[s + 1] : (long long)d + 1;
         auto enter_segment = [&]() {
@@ -395,7 +415,8 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         // run's first kSfLocal segments are collected in shared memory and go out after the last
         // row; later segments go to the global counters directly.  No warp waits for another.
         auto leave_segment = [&](int64_t e) {
-            if (counted) {
+            // a short segment lies in a few warps only: the others have counted nothing
+            if (counted && __any_sync(0xffffffffu, dirty)) {
                 const int li = s - s_first;
 #pragma unroll
                 for (int j = 0; j < kNumCand; ++j) {
@@ -407,6 +428,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     }
                 }
             }
+            dirty = false;
             s = seg_advance(sh.off, S_use, s + 1, e);
             send = s < S_use ? sh.off[s + 1] : (long long)d + 1;
             enter_segment();
@@ -451,6 +473,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     row_x(r, x, one);
                     if (one) count_float4(x, any_neg ? 0x10000u : (unsigned int)trow[r * kFusedWarps], cs, tier, acc);
                 }
+                dirty = true;  // (rows were counted, or the loop did not run and it does not matter)
             } else {
                 // nothing to count here, but the ring keeps turning
                 for (; r < pure_end; ++r) {
@@ -473,10 +496,12 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 if (re1 > rows_hi) re1 = rows_hi;
                 const int64_t e0 = (lo4 + (int64_t)r * kRowF4 + tid) << 2;
                 const float xx[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
+                const int64_t we0 = re0 + 128 * w;  // this warp's 128 elements of the row
                 int64_t cur = re0;
                 while (cur < re1 && s < S_use) {
                     const int64_t seg_hi = send < re1 ? send : re1;
-                    if (one && counted) {
+                    if (one && counted && we0 < seg_hi && we0 + 128 > cur) {
+                        dirty = true;
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
                             const int64_t e = e0 + t;
@@ -502,6 +527,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 if (owns_tail && counted && tail_i >= cur && tail_i < seg_hi) {
 #pragma unroll
                     for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
+                    dirty = true;
                 }
                 cur = seg_hi;
                 if (send <= d) leave_segment(cur); else break;
@@ -515,11 +541,13 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             if (x && q < S_use) atomicAdd(&v.counts[(size_t)q * kNumCand + j % kNumCand], (unsigned long long)x);
         }
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
+        stamp(5);
         if (!grid_barrier(&bars[1], (unsigned)G, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
         if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
+        stamp(6);
     }
 
     // ------------------------------------------------------------------ resolve
@@ -534,7 +562,11 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             unsigned long long nz = 0ull;
             if (!bad && n > 0) {
                 if (sh.counted[q]) {
-                    const Alg1Path p = alg1_replay(v.counts + (size_t)q * kNumCand, kk);
+                    // the ten counts come in together; the rounds are then replayed on the copy
+                    unsigned long long cnt[kNumCand];
+#pragma unroll
+                    for (int j = 0; j < kNumCand; ++j) cnt[j] = __ldcg(&v.counts[(size_t)q * kNumCand + j]);
+                    const Alg1Path p = alg1_replay(cnt, kk);
                     float t = INFINITY;
                     for (int j = 0; j < kNumCand; ++j) if (sh.ord[q][j] == p.chosen) t = sh.cs[q][j];
                     sh.thr[q] = t;
@@ -542,7 +574,6 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 } else {
                     nz = (unsigned long long)n;  // everything selected
                 }
-                if (c == 0) alg1_resolve(seg_state_of(v, q), kk);
             }
             if (c == 0 && seg_nnz_out) seg_nnz_out[q] = (int64_t)nz;
             my_nnz += nz;
@@ -579,6 +610,12 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         };
         // survivors of the float4 at element index e0, starting the segment walk at sx
         auto mask_of = [&](const float4 x, int64_t e0, int sx) -> unsigned int {
+            while (sx < S_use && sh.off[sx + 1] <= e0) ++sx;
+            if (sx < S_use && sh.off[sx + 1] >= e0 + 4) {  // the four elements share a segment
+                const float t = sh.thr[sx];
+                return (unsigned)(fabsf(x.x) > t) | ((unsigned)(fabsf(x.y) > t) << 1) |
+                       ((unsigned)(fabsf(x.z) > t) << 2) | ((unsigned)(fabsf(x.w) > t) << 3);
+            }
             unsigned int m = 0u;
             m |= (unsigned)(fabsf(x.x) > thr_at(sx, e0));
             m |= (unsigned)(fabsf(x.y) > thr_at(sx, e0 + 1)) << 1;
@@ -611,13 +648,15 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         };
         // step 0: which (row, warp) segments of 128 elements can hold a survivor: all of one
         // layer-segment, the recorded maximum decides; with a boundary inside, always read
+        const int s_run = seg_find(sh.off, S_use, run_lo);  // the segment the run starts in
+        int su0 = s_run;                                     // this lane's walk through the segments
         for (int r = lane; r < nrows; r += 32) {
             const int64_t ue0 = ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w;
             int64_t ue1 = ue0 + 128;
             if (ue1 > (hi4 << 2)) ue1 = hi4 << 2;
             bool ql = false;
             if (ue0 < ue1) {
-                const int su = seg_find(sh.off, S_use, ue0);
+                const int su = su0 = seg_advance(sh.off, S_use, su0, ue0);
                 if (su < S_use) {
                     if (sh.off[su + 1] >= ue1) {
                         const float t = sh.thr[su];
@@ -630,7 +669,9 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             table[r * kFusedWarps + w] = ql ? kSfPending : (unsigned short)0;
         }
         __syncwarp();
-        // step 1: survivors of every qualifying segment into the table
+        // step 1: survivors of every qualifying segment into the table (rows come in ascending
+        // order, so the warp's position among the segments only moves forward)
+        int su1 = s_run;
         for (int cursor = 0; cursor < nrows;) {
             const int n = gather(cursor, true);
             float4 x[kSfGroupRows];
@@ -649,7 +690,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     const int r = sh.qrow[w][q];
                     const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
                     // every lane starts its walk at the segment of the warp's first element
-                    const int su = seg_find(sh.off, S_use, ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w);
+                    const int su = su1 = seg_advance(sh.off, S_use, su1, ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w);
                     const unsigned int cnt =
                         __reduce_add_sync(0xffffffffu, i < hi4 ? __popc(mask_of(x[q], i << 2, su)) : 0u);
                     if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
@@ -658,7 +699,8 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             __syncwarp();
         }
         __syncthreads();
-        // step 2: survivors per row (thread t takes row t) to the row's word in global memory
+        // step 2: survivors per row (thread t takes row t), a scan over this run's rows, and the
+        // run's total to this CTA's word in global memory
         unsigned int mine_row = 0u;
         if (tid < nrows) {
             const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
@@ -668,22 +710,9 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 mine_row += (y.x & 0xffffu) + (y.x >> 16) + (y.y & 0xffffu) + (y.y >> 16) +
                             (y.z & 0xffffu) + (y.z >> 16) + (y.w & 0xffffu) + (y.w >> 16);
             }
-            rowcnt[(int64_t)c * rows_per_cta + tid] = mine_row;
         }
-        if (!grid_barrier(&bars[3], (unsigned)G, &sh.ok)) {
-            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
-            goto leave;
-        }
-        // survivors in the runs before this one (integers: any order), then a scan over this run
+        unsigned int run_total;
         {
-            unsigned long long before = 0ull;
-            const int64_t R0 = (int64_t)c * rows_per_cta;
-            for (int64_t R = tid; R < R0; R += kFusedThreads) before += __ldcg(rowcnt + R);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-            if (tid == 0) sh.total = 0ull;
-            __syncthreads();
-            if (lane == 0 && before) atomicAdd(&sh.total, before);
             unsigned int sc = mine_row;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -700,11 +729,25 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                 if (lane >= o) y += t;
             }
             const unsigned int wpre = __shfl_sync(0xffffffffu, y - y0, w);
-            const unsigned int run_total = __shfl_sync(0xffffffffu, y, 31);
+            run_total = __shfl_sync(0xffffffffu, y, 31);
             if (tid < nrows) sh.rowpre[tid] = wpre + sc - mine_row;
+            if (tid == 0) { cta_tot[c] = run_total; sh.total = 0ull; }
+        }
+        if (!grid_barrier(&bars[3], (unsigned)G, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        // survivors in the runs before this one (integers: any order): thread t reads CTA t's word
+        {
+            unsigned long long before = 0ull;
+            for (int t = tid; t < c; t += kFusedThreads) before += __ldcg(cta_tot + t);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+            if (lane == 0 && before) atomicAdd(&sh.total, before);
             __syncthreads();
             const unsigned long long base = sh.total;
             // step 3: every warp writes the survivors of its segments that have any
+            int su3 = s_run;
             for (int cursor = 0; cursor < nrows;) {
                 const int n = gather(cursor, false);
                 float4 x[kSfGroupRows];
@@ -722,7 +765,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     if (q >= n) continue;
                     const int r = sh.qrow[w][q];
                     const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-                    const int su = seg_find(sh.off, S_use, ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w);
+                    const int su = su3 = seg_advance(sh.off, S_use, su3, ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w);
                     const unsigned int m = i < hi4 ? mask_of(x[q], i << 2, su) : 0u;
                     const unsigned int earlier =
                         __reduce_add_sync(0xffffffffu, lane < w ? (unsigned int)table[r * kFusedWarps + lane] : 0u);
@@ -768,7 +811,28 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             }
         }
     }
+    // CTA 0 completes the records that the host can read back, off everybody's way
+    if (c == 0 && !bad) {
+        for (int q = tid; q < S; q += kFusedThreads) {
+            const long long n = sh.off[q + 1] - sh.off[q];
+            if (n <= 0 || !sh.counted[q]) continue;
+            long long kk = seg_k[q];
+            if (kk > n) kk = n;
+            unsigned long long cnt[kNumCand];
+#pragma unroll
+            for (int j = 0; j < kNumCand; ++j) cnt[j] = __ldcg(&v.counts[(size_t)q * kNumCand + j]);
+            gk_stats rec = v.stats[q];
+            const Alg1Path p = alg1_replay(cnt, kk);
+            for (int r = 0; r < p.rounds; ++r) rec.counts[r] = p.est[r];
+            rec.rounds = p.rounds;
+            rec.thr_final = v.cand64[(size_t)q * kNumCand + p.chosen];
+            rec.nnz = p.est[p.rounds - 1];
+            v.stats[q] = rec;
+            v.thr_sel[q] = sh.thr[q];
+        }
+    }
     if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
+    stamp(7);
 
 leave:
     // the CTA that leaves last clears the barrier counters for the next call
@@ -778,7 +842,7 @@ leave:
         const unsigned int t = atomicAdd(&bars[2], 1u);
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[6] = global_timer_ns();
-            bars[0] = 0u; bars[1] = 0u; bars[3] = 0u;
+            bars[0] = 0u; bars[1] = 0u; bars[3] = 0u; bars[4] = 0u;
             __threadfence();
             bars[2] = 0u;
         }
@@ -843,20 +907,22 @@ int enqueue_gk_fused_seg(Workspace* ws, const float* g, float* eps, int64_t d, c
     int S_arg = (int)S;
     Ctrl* ctrl = ws->ctrl;
     SegScratch v = segmented_views(ws);
-    unsigned int* bars = ws->bars + 10;  // counters 10..13: three barriers and the exit
-    unsigned int* rowcnt = ws->rowcnt;
+    unsigned int* bars = ws->bars + 10;  // counters 10..14: three barriers, the exit, the quantile ticket
+    unsigned int* cta_tot = ws->cta_counts;  // one word per CTA: the survivors of its run
     int64_t cap = output_capacity(d);
+    unsigned long long* trace = ws->cta_trace;
     void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&seg_offsets, (void*)&seg_k, (void*)&S_arg,
-                    (void*)&rpc, (void*)&u_slots, (void*)&ctrl, (void*)&v, (void*)&bars, (void*)&rowcnt,
-                    (void*)&idx_out, (void*)&val_out, (void*)&seg_nnz_out, (void*)&nnz_out, (void*)&cap};
-    static_assert(sizeof(args) / sizeof(args[0]) == 17, "k_gk_fused_seg takes 17 arguments");
+                    (void*)&rpc, (void*)&u_slots, (void*)&ctrl, (void*)&v, (void*)&bars, (void*)&cta_tot,
+                    (void*)&idx_out, (void*)&val_out, (void*)&seg_nnz_out, (void*)&nnz_out, (void*)&cap,
+                    (void*)&trace};
+    static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused_seg takes 18 arguments");
     stage_mark(ws, st, 0);
     GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused_seg, dim3((unsigned)G), dim3(kFusedThreads), args,
                                             smem, st));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_grid = (int)G;
-    ws->last_fused = false;
+    ws->last_fused = true;  // the per-CTA trace is this kernel's
     ws->phase_spans = 6;
     return GK_OK;
 }
