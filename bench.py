@@ -39,9 +39,9 @@ UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
 N_ROTATE = 20   # distinct gradients: the workload's 20 error-compensation iterations, then again
 EPISODE = 20    # steps that share one residual buffer (eps starts at zero)
-# DRAM bytes of one k_gk_fused launch at d = 25,557,032 (258.6 MB read + 78.3 MB written), from the
+# DRAM bytes of one k_gk_fused launch at d = 25,557,032 (260.6 MB read + 78.7 MB written), from the
 # ncu capture summarised under profiles/; valid only for the kernel as it stood at that capture
-FUSED_DRAM_BYTES_PER_LAUNCH = 336867584
+FUSED_DRAM_BYTES_PER_LAUNCH = 339367424
 FUSED_DRAM_CAPTURE_D = 25557032
 MAX_EPS = 48    # residual buffers kept (pre-zeroed); beyond that they are reused as they stand
 
@@ -251,6 +251,24 @@ def run_ours(args):
 
     def step(t):
         gk.gk_sparsify(gs[t % n_rot], epss[(t // EPISODE) % n_eps], k, idx, val, nnz)
+
+    if args.call != "gk":
+        # a capture of one of the other entry points: the same loop, nothing else (--loop-only)
+        if args.call == "segmented":
+            part = w.partition
+            d_off = torch.from_numpy(part.offsets).to(dev)
+            d_k = torch.from_numpy(part.seg_k(*wl.RHO[rho])).to(dev)
+            seg_nnz = torch.zeros(part.S, dtype=torch.int64, device=dev)
+
+            def step(t):  # noqa: F811
+                gk.gk_sparsify_segmented(gs[t % n_rot], epss[(t // EPISODE) % n_eps], d_off, d_k, idx, val,
+                                         seg_nnz, nnz)
+        elif args.call == "topk_sparsify":
+            def step(t):  # noqa: F811
+                gk.topk_sparsify(gs[t % n_rot], epss[(t // EPISODE) % n_eps], k, idx, val, nnz)
+        else:
+            def step(t):  # noqa: F811
+                gk.topk_exact(gs[t % n_rot], k, idx, val)
 
     def barrier():
         torch.cuda.synchronize()
@@ -537,9 +555,13 @@ def main():
                     help="number of gradient buffers kept on the device (default 20; small for captures)")
     ap.add_argument("--loop-only", action="store_true",
                     help="run only warm-up and the timed loop (for profiler captures)")
+    ap.add_argument("--call", default="gk", choices=["gk", "segmented", "topk_exact", "topk_sparsify"],
+                    help="entry point the timed loop calls (other than gk: with --loop-only, for captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every workload family (Gaussian_k, segmented, exact Top_k) and print one line each")
     args = ap.parse_args()
+    if args.call != "gk" and not args.loop_only:
+        ap.error("--call other than gk needs --loop-only")
     if args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

@@ -227,21 +227,28 @@ int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out);
  * While enabled, every call records a CUDA event on its stream before its first
  * kernel and after each kernel.  gk_last_stage_ms synchronises the stream and
  * writes the durations in milliseconds of the stages of the last call enqueued on
- * it to HOST ms_out[0..*n_stages-1] (at most 8).  gk_sparsify, fused kernel: the
- * kernel, then six spans from timestamps the kernel takes itself (accumulate incl.
- * first barrier, counting loop, second barrier, replay of the rounds, compaction,
- * exit of the last CTA); three-kernel path: accumulate, count, compact.  topk_exact:
- * three histogram passes and compact; topk_sparsify has accumulate first.
+ * it to HOST ms_out[0..*n_stages-1] (at most 8).  Single-kernel forms: the kernel,
+ * then spans between timestamps the kernel takes itself (CTA 0 and the CTA that
+ * leaves last).  gk_sparsify and gk_sparsify_segmented: accumulate incl. first
+ * barrier and thresholds, counting loop, second barrier, replay of the rounds,
+ * compaction, exit of the last CTA.  topk_exact and topk_sparsify: first pass,
+ * barrier and first digit, second pass to second digit, third pass to third digit,
+ * counts and fourth barrier, offsets and write-out, exit of the last CTA.
+ * Multi-kernel forms, one value per kernel: accumulate, count, compact; for
+ * Top_k three histogram passes and compact, with accumulate first in topk_sparsify.
  */
 int gk_stage_timing(int enable);
 int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages);
 
 /*
- * Per-CTA trace of the last fused gk_sparsify call on `stream` (tracing aid).
- * Synchronises the stream and writes 8 uint64 per CTA to HOST host_out (room for
- * 512 x 8): %globaltimer in ns at the CTA's start, before and after the first
- * grid barrier, before and after the second, and at its end (slots 6, 7 unused).
- * *n_ctas receives the number of CTAs, 0 if the last call did not run that kernel.
+ * Per-CTA trace of the last single-kernel gk_sparsify or gk_sparsify_segmented
+ * call on `stream` (tracing aid).  Synchronises the stream and writes 8 uint64
+ * per CTA to HOST host_out (room for 512 x 8), %globaltimer in ns.  gk_sparsify:
+ * the CTA's start, before and after the first grid barrier, before and after the
+ * second, before and after the third, its end.  gk_sparsify_segmented: start,
+ * table read, end of the first phase, after the first barrier, thresholds formed,
+ * end of the counting, after the second barrier, end.
+ * *n_ctas receives the number of CTAs, 0 if the last call did not run such a kernel.
  */
 int gk_last_cta_trace(gk_stream_t stream, uint64_t* host_out, int* n_ctas);
 
