@@ -21,6 +21,7 @@
 //   * the comparison |u_i| > thres is taken in fp64 (u_i widened exactly).
 //   * k >= d (p <= 0): every element is selected, no statistics.
 //   * exact Top_k breaks ties of equal magnitude toward the lower index.
+//   * DGC_k (one sentence in the paper): see the comment at oracle_dgck_select.
 //
 // Pins (tests that do not pass through this file's own formulas): see
 // tests/test_oracle_pins.py.  Nothing here is "parity unpinned".
@@ -239,6 +240,58 @@ double oracle_error_ratio(const float* u, int64_t d, const int32_t* idx, int64_t
     for (int64_t i = 0; i < d; ++i) all += (double)u[i] * (double)u[i];
     for (int64_t j = 0; j < nnz; ++j) kept += (double)u[idx[j]] * (double)u[idx[j]];
     return (all - kept) / all;
+}
+
+// ---------------------------------------------------------------------------
+// DGC_k, the hierarchical sampling selector the paper compares against
+// (Section 3.3: "sample only 0.1% to 1% of the gradients to estimate the
+// threshold hierarchically", with two top-k selections on subsets of the
+// vector; Section 4.3: a 1% sample).  The paper gives no more than that; the
+// reading taken here:
+//   1. the sample is the multiset { |u[s_j]| : j < m } at the positions s_j the
+//      caller drew (the random draw is an input, not part of the arithmetic);
+//   2. first top-k, on the sample: with k_m = ceil(k * m / d) (the density k/d
+//      applied to the sample size), tau = the k_m-th largest sampled magnitude;
+//   3. candidates C = { i : |u_i| >= tau } over the whole vector;
+//   4. second top-k, on C, only when |C| > k: the k largest magnitudes of C,
+//      ties toward the lower index; otherwise all of C is returned (fewer than
+//      k entries are accepted, as with any sampled threshold).
+// Pairs come out in ascending index.  info: [0] bits of tau, [1] |C|, [2] k_m.
+// Returns the number of pairs.
+// ---------------------------------------------------------------------------
+int64_t oracle_dgck_select(const float* u, int64_t d, int64_t k, const int32_t* sidx, int64_t m,
+                           int32_t* idx, float* val, int64_t* info) {
+    std::vector<float> v((size_t)m);
+    for (int64_t j = 0; j < m; ++j) v[(size_t)j] = std::fabs(u[sidx[j]]);        // step 1
+    const int64_t km = (k * m + d - 1) / d;                                       // step 2
+    std::sort(v.begin(), v.end(), [](float a, float b) { return a > b; });
+    const float tau = v[(size_t)(km - 1)];
+    std::vector<int32_t> cand;                                                    // step 3
+    for (int64_t i = 0; i < d; ++i)
+        if (std::fabs(u[i]) >= tau) cand.push_back((int32_t)i);
+    const int64_t n = (int64_t)cand.size();
+    uint32_t tb;
+    std::memcpy(&tb, &tau, 4);
+    info[0] = (int64_t)tb; info[1] = n; info[2] = km;
+    if (n > k) {                                                                  // step 4
+        std::stable_sort(cand.begin(), cand.end(), [&](int32_t a, int32_t b) {
+            return std::fabs(u[a]) > std::fabs(u[b]);   // stable: equal magnitudes keep index order
+        });
+        cand.resize((size_t)k);
+        std::sort(cand.begin(), cand.end());
+    }
+    for (size_t j = 0; j < cand.size(); ++j) { idx[j] = cand[j]; val[j] = u[cand[j]]; }
+    return (int64_t)cand.size();
+}
+
+// Eq. 2 with Comp_k = DGC_k: u = g + eps, selection as above, eps <- u - Comp(u).
+int64_t oracle_dgck_sparsify(const float* g, float* eps, int64_t d, int64_t k, const int32_t* sidx,
+                             int64_t m, int32_t* idx, float* val, int64_t* info) {
+    std::vector<float> u((size_t)d);
+    oracle_accumulate(g, eps, d, u.data());
+    const int64_t n = oracle_dgck_select(u.data(), d, k, sidx, m, idx, val, info);
+    oracle_residual(u.data(), d, idx, val, n, eps);
+    return n;
 }
 
 }  // extern "C"

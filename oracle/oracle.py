@@ -81,6 +81,10 @@ def lib() -> C.CDLL:
         L.oracle_topk_exact.restype = None
         L.oracle_error_ratio.argtypes = [fp, C.c_int64, ip, C.c_int64]
         L.oracle_error_ratio.restype = C.c_double
+        L.oracle_dgck_select.argtypes = [fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
+        L.oracle_dgck_select.restype = C.c_int64
+        L.oracle_dgck_sparsify.argtypes = [fp, fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
+        L.oracle_dgck_sparsify.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -187,3 +191,37 @@ def topk_exact(u: np.ndarray, k: int) -> Tuple[np.ndarray, np.ndarray]:
 def error_ratio(u: np.ndarray, idx: np.ndarray) -> float:
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     return lib().oracle_error_ratio(_f(u), u.shape[0], _i(idx), idx.shape[0])
+
+
+@dataclass
+class DgcInfo:
+    tau_bits: int   # fp32 pattern of the sampled threshold
+    n_cand: int     # entries of the vector at or above it
+    k_m: int        # rank taken in the sample
+
+    @property
+    def tau(self) -> float:
+        return float(np.array([self.tau_bits], dtype=np.uint32).view(np.float32)[0])
+
+
+def dgck_select(u: np.ndarray, k: int, sample_idx: np.ndarray):
+    """DGC_k on a given vector.  Returns (idx, val, DgcInfo)."""
+    d = u.shape[0]
+    sample_idx = np.ascontiguousarray(sample_idx, dtype=np.int32)
+    idx = np.empty(d, dtype=np.int32)
+    val = np.empty(d, dtype=np.float32)
+    info = np.zeros(3, dtype=np.int64)
+    n = lib().oracle_dgck_select(_f(u), d, k, _i(sample_idx), sample_idx.shape[0], _i(idx), _f(val), _l(info))
+    return idx[:n].copy(), val[:n].copy(), DgcInfo(int(info[0]), int(info[1]), int(info[2]))
+
+
+def dgck_sparsify(g: np.ndarray, eps: np.ndarray, k: int, sample_idx: np.ndarray):
+    """One step of Eq. 2 with DGC_k.  eps is updated IN PLACE.  Returns (idx, val, DgcInfo)."""
+    d = g.shape[0]
+    sample_idx = np.ascontiguousarray(sample_idx, dtype=np.int32)
+    idx = np.empty(d, dtype=np.int32)
+    val = np.empty(d, dtype=np.float32)
+    info = np.zeros(3, dtype=np.int64)
+    n = lib().oracle_dgck_sparsify(_f(g), _f(eps), d, k, _i(sample_idx), sample_idx.shape[0], _i(idx), _f(val),
+                                   _l(info))
+    return idx[:n].copy(), val[:n].copy(), DgcInfo(int(info[0]), int(info[1]), int(info[2]))

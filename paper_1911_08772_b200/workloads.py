@@ -38,6 +38,7 @@ TAG_SWEEP_NORMAL = 5
 TAG_SWEEP_LAPLACE = 6
 TAG_PARTITION = 7
 TAG_MISC = 8
+TAG_SAMPLE = 9
 
 
 def ceil_k(d: int, num: int, den: int) -> int:
@@ -277,3 +278,16 @@ def sweep_point(d: int, dist: str) -> Workload:
 def misc_rng(stream: int) -> np.random.Generator:
     """Generator for small hand-shaped test vectors."""
     return _rng(TAG_MISC, 0, stream, MASTER_SEED)
+
+
+def sample_positions(d: int, m: int, step: int = 0, seed: int = MASTER_SEED) -> np.ndarray:
+    """m positions drawn uniformly from [0, d) with replacement (int32): the random sample a
+    sampling selector such as DGC_k takes.  The draw is an input of the method, so it is made
+    here and handed to whoever needs it."""
+    rng = _rng(TAG_SAMPLE, 0, step, seed)
+    return rng.integers(0, d, size=m, dtype=np.int64).astype(np.int32)
+
+
+def sample_size(d: int, num: int = 1, den: int = 100) -> int:
+    """Sample size ceil(d * num / den); the default is the 1 % sample of Section 4.3."""
+    return max(1, (d * num + den - 1) // den)

@@ -411,3 +411,109 @@ def test_eq5_ratio_from_sorted_normalised_magnitudes():
     pi = np.sort(np.abs(u.astype(np.float64)) / np.abs(u).max())[::-1]
     ratio = (pi[k:] ** 2).sum() / (pi ** 2).sum()
     assert abs(orc.error_ratio(u, idx) - ratio) < 1e-12
+
+
+# --------------------------------------------------------------------------- DGC_k (Section 3.3)
+def _dgck_brute(u, k, sidx):
+    """Pure-Python DGC_k: sampled threshold, candidates, second selection with ties to the
+    lower index."""
+    d = len(u)
+    mags = sorted((abs(float(u[j])) for j in sidx), reverse=True)
+    km = -(-k * len(sidx) // d)
+    tau = mags[km - 1]
+    cand = [i for i in range(d) if abs(float(u[i])) >= tau]
+    n = len(cand)
+    if n > k:
+        cand = sorted(sorted(cand, key=lambda i: (-abs(float(u[i])), i))[:k])
+    return cand, tau, n, km
+
+
+def test_dgck_hand_worked_cases():
+    lines = [l.split() for l in open(os.path.join(GOLDEN, "dgck_hand_case.txt")) if not l.startswith("#")]
+    u = np.array([float(x) for x in lines[0][1:]], dtype=np.float32)
+    for l in lines[1:]:
+        assert l[0] == "case"
+        k = int(l[l.index("k") + 1])
+        s0, t0, i0 = l.index("sample"), l.index("tau"), l.index("idx")
+        sidx = np.array([int(x) for x in l[s0 + 1:t0]], dtype=np.int32)
+        tau, n, km = float(l[t0 + 1]), int(l[l.index("n") + 1]), int(l[l.index("km") + 1])
+        want = np.array([int(x) for x in l[i0 + 1:]], dtype=np.int32)
+        idx, val, info = orc.dgck_select(u, k, sidx)
+        assert (info.tau, info.n_cand, info.k_m) == (tau, n, km), l[1]
+        assert np.array_equal(idx, want) and np.array_equal(val, u[want]), l[1]
+
+
+def test_dgck_brute_force_small_inputs_with_ties():
+    rng = wl.misc_rng(40)
+    for trial in range(300):
+        d = int(rng.integers(1, 40))
+        k = int(rng.integers(1, d + 1))
+        m = int(rng.integers(1, 2 * d + 1))
+        # few distinct magnitudes, both signs, zeros: ties everywhere
+        u = (rng.integers(-4, 5, size=d) * 0.5).astype(np.float32)
+        if trial % 3 == 0:
+            u = rng.standard_normal(d).astype(np.float32)
+        sidx = rng.integers(0, d, size=m).astype(np.int32)
+        idx, val, info = orc.dgck_select(u, k, sidx)
+        cand, tau, n, km = _dgck_brute(u, k, sidx)
+        assert (info.tau, info.n_cand, info.k_m) == (tau, n, km)
+        assert idx.tolist() == cand and np.array_equal(bits(val), bits(u[cand]))
+
+
+def test_dgck_with_the_whole_vector_as_sample_is_exact_topk():
+    # sampling every position once makes k_m = k and tau the k-th largest magnitude, so the
+    # candidates hold the exact Top_k and the second selection returns it (numpy route)
+    rng = wl.misc_rng(41)
+    for d, k in [(1000, 1), (1000, 10), (4097, 333), (50_000, 50)]:
+        u = rng.standard_normal(d).astype(np.float32)
+        u[rng.integers(0, d, size=d // 10)] = np.float32(1.25)  # planted ties
+        sidx = rng.permutation(d).astype(np.int32)
+        idx, val, info = orc.dgck_select(u, k, sidx)
+        order = np.lexsort((np.arange(d), -np.abs(u).astype(np.float64)))  # magnitude desc, index asc
+        want = np.sort(order[:k]).astype(np.int32)
+        assert info.k_m == k and info.n_cand >= k
+        assert np.array_equal(idx, want) and np.array_equal(bits(val), bits(u[want]))
+
+
+def test_dgck_properties_on_workload_like_inputs():
+    d = 1 << 20
+    for dist, rho in [("normal", "1e-3"), ("laplace", "1e-2"), ("normal", "1e-2")]:
+        w = wl.sweep_point(d, dist)
+        u = w.grad(0)
+        k = wl.ceil_k(d, *wl.RHO[rho])
+        sidx = wl.sample_positions(d, wl.sample_size(d), step=3)
+        idx, val, info = orc.dgck_select(u, k, sidx)
+        mag = np.abs(u)
+        tau = np.float32(info.tau)
+        assert info.k_m == -(-k * sidx.size // d)
+        # tau is the k_m-th largest sampled magnitude (numpy partition)
+        sm = mag[sidx]
+        assert tau == np.partition(sm, sm.size - info.k_m)[sm.size - info.k_m]
+        assert info.n_cand == int((mag >= tau).sum())
+        assert np.all(np.diff(idx) > 0) and np.array_equal(bits(val), bits(u[idx]))
+        if info.n_cand <= k:
+            assert np.array_equal(idx, np.nonzero(mag >= tau)[0])
+        else:
+            # more candidates than k: the answer is the exact Top_k of the whole vector
+            kth = np.partition(mag, d - k)[d - k]
+            assert idx.size == k and mag[idx].min() == kth and int((mag > kth).sum()) <= k
+            assert set(np.nonzero(mag > kth)[0]).issubset(set(idx.tolist()))
+        # a 1 % sample estimates the density within sampling noise (binomial, k_m entries)
+        assert abs(info.n_cand / k - 1.0) < 6.0 / math.sqrt(info.k_m)
+
+
+def test_dgck_sparsify_identity():
+    rng = wl.misc_rng(42)
+    d, k = 20_000, 100
+    g = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    e = (rng.standard_normal(d) * 2e-3).astype(np.float32)
+    sidx = wl.sample_positions(d, 2000, step=5)
+    u = g + e
+    eps = e.copy()
+    idx, val, info = orc.dgck_sparsify(g, eps, k, sidx)
+    i2, v2, info2 = orc.dgck_select(u, k, sidx)
+    assert np.array_equal(idx, i2) and np.array_equal(bits(val), bits(v2)) and info == info2
+    comp = np.zeros(d, dtype=np.float32)
+    comp[idx] = val
+    assert np.array_equal(bits(comp + eps), bits(u + np.float32(0)))  # Comp(u) + eps_new == u
+    assert np.all(eps[idx] == 0) and np.array_equal(bits(np.delete(eps, idx)), bits(np.delete(u, idx)))
