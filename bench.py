@@ -266,6 +266,14 @@ def run_ours(args):
         elif args.call == "topk_sparsify":
             def step(t):  # noqa: F811
                 gk.topk_sparsify(gs[t % n_rot], epss[(t // EPISODE) % n_eps], k, idx, val, nnz)
+        elif args.call in ("dgck_sparsify", "dgck_select"):
+            smp = torch.from_numpy(wl.sample_positions(d, wl.sample_size(d), step=0)).to(dev)
+            if args.call == "dgck_sparsify":
+                def step(t):  # noqa: F811
+                    gk.dgck_sparsify(gs[t % n_rot], epss[(t // EPISODE) % n_eps], k, smp, idx, val, nnz)
+            else:
+                def step(t):  # noqa: F811
+                    gk.dgck_select(gs[t % n_rot], k, smp, idx, val, nnz)
         else:
             def step(t):  # noqa: F811
                 gk.topk_exact(gs[t % n_rot], k, idx, val)
@@ -389,7 +397,43 @@ def run_ours(args):
         topk[name] = rec
     gk.gk_set_path(0)
     ms_topk, ms_topk_sp = topk["fused"]["topk_exact_ms"], topk["fused"]["topk_sparsify_ms"]
-    del eps2, us
+
+    # ---- DGC_k (the paper's third operator, Section 4.3: a 1 % sample) on the same data, as
+    # operator and as sparsifier; a fresh seeded sample per step, resident on the device
+    smps = [torch.from_numpy(wl.sample_positions(d, wl.sample_size(d), step=j)).to(dev) for j in range(4)]
+    for t in range(3):
+        gk.dgck_select(us[t % len(us)], k, smps[t % 4], tk_idx, tk_val, nnz)
+    ms_dg_op = time_region(torch, lambda t: gk.dgck_select(us[t % len(us)], k, smps[t % 4], tk_idx, tk_val, nnz),
+                           Kt) / Kt
+    eps2.zero_()
+    for t in range(3):
+        gk.dgck_sparsify(gs[t % n_rot], eps2, k, smps[t % 4], tk_idx, tk_val, nnz)
+    ms_dg_sp = time_region(torch, lambda t: gk.dgck_sparsify(gs[t % n_rot], eps2, k, smps[t % 4], tk_idx, tk_val,
+                                                             nnz), Kt) / Kt
+    gk.gk_stage_timing(True)
+    acc_op, acc_sp = np.zeros(8), np.zeros(8)
+    for t in range(20):
+        gk.dgck_select(us[t % len(us)], k, smps[t % 4], tk_idx, tk_val, nnz)
+        acc_op += np.array(gk.gk_last_stage_ms()[:8])
+        gk.dgck_sparsify(gs[t % n_rot], eps2, k, smps[t % 4], tk_idx, tk_val, nnz)
+        acc_sp += np.array(gk.gk_last_stage_ms()[:8])
+    gk.gk_stage_timing(False)
+    dg_info = gk.dgck_last_info()
+    dg_names = ["kernel", "sample_threshold", "stream", "barrier+count", "second_selection", "count+barrier",
+                "offsets+emit", "last_cta_exit"]
+    m_s = int(smps[0].numel())
+    dgck = {"sample": f"{m_s} positions (1 % of d), uniform with replacement, seeded",
+            "dgck_select_ms": ms_dg_op, "dgck_sparsify_ms": ms_dg_sp,
+            "dgck_select_gbs_4B_per_elem": (4.0 * d + 32.0 * m_s + 8.0 * k) / ms_dg_op / 1e6,
+            "dgck_sparsify_gbs_12B_per_elem": (12.0 * d + 64.0 * m_s + 12.0 * k) / ms_dg_sp / 1e6,
+            "vs_gaussiank_sparsify": ms_dg_sp / (ms / K), "vs_topk_sparsify": ms_dg_sp / ms_topk_sp,
+            "candidates_last": dg_info[1], "k_m": dg_info[2], "pairs_last": dg_info[3],
+            "phase_ms_operator": dict(zip(dg_names, (acc_op / 20).tolist())),
+            "phase_ms_sparsifier": dict(zip(dg_names, (acc_sp / 20).tolist())),
+            "note": "algorithmic bytes: one pass over the vector (4 d, or 12 d with the add and the store of "
+                    "u), one 32-byte sector per sampled position and operand, 8 bytes per pair (+4 per "
+                    "cleared slot)"}
+    del eps2, us, smps
 
     # ---- the error ratio of Eq. 5 for one Gaussian_k step and one Top_k step from eps = 0
     diag = {"bound_eq4_1_minus_k_over_d": 1.0 - k / d, "bound_theorem1_squared": (1.0 - k / d) ** 2}
@@ -458,7 +502,7 @@ def run_ours(args):
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
                  "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
-        "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
+        "dgck": dgck, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
         "clocks": sampler.summary(),
     }
     print(json.dumps(line))
@@ -534,9 +578,16 @@ def run_sweep(args):
                 gk.topk_exact(u, k, tk_i, tk_v)
             ms_tk = time_region(torch, lambda t: gk.topk_exact(u, k, tk_i, tk_v), 10) / 10
             ms_tks = timed(lambda t: gk.topk_sparsify(gs[t % n_grad], eps, k, tk_i, tk_v, nnz))
+            smp = torch.from_numpy(wl.sample_positions(d, wl.sample_size(d), step=0)).to(dev)
+            for _ in range(3):
+                gk.dgck_select(u, k, smp, tk_i, tk_v, nnz)
+            ms_dg = time_region(torch, lambda t: gk.dgck_select(u, k, smp, tk_i, tk_v, nnz), 10) / 10
+            ms_dgs = timed(lambda t: gk.dgck_sparsify(gs[t % n_grad], eps, k, smp, tk_i, tk_v, nnz))
             rec.update({"topk_exact_ms": ms_tk, "topk_sparsify_ms": ms_tks,
                         "speedup_vs_topk_sparsify": ms_tks / ms_gk,
-                        "topk_exact_gbs_12B_per_elem": 12.0 * d / ms_tk / 1e6})
+                        "topk_exact_gbs_12B_per_elem": 12.0 * d / ms_tk / 1e6,
+                        "dgck_select_ms": ms_dg, "dgck_sparsify_ms": ms_dgs,
+                        "dgck_candidates_last": gk.dgck_last_info()[1]})
             print(json.dumps(rec), flush=True)
         del gs, eps, idx, val
         torch.cuda.empty_cache()
@@ -555,7 +606,7 @@ def main():
                     help="number of gradient buffers kept on the device (default 20; small for captures)")
     ap.add_argument("--loop-only", action="store_true",
                     help="run only warm-up and the timed loop (for profiler captures)")
-    ap.add_argument("--call", default="gk", choices=["gk", "segmented", "topk_exact", "topk_sparsify"],
+    ap.add_argument("--call", default="gk", choices=["gk", "segmented", "topk_exact", "topk_sparsify", "dgck_select", "dgck_sparsify"],
                     help="entry point the timed loop calls (other than gk: with --loop-only, for captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every workload family (Gaussian_k, segmented, exact Top_k) and print one line each")

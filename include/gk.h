@@ -49,6 +49,7 @@ typedef enum gk_status {
 #define GK_DEV_TRUNCATED 1    /* more survivors than the output capacity */
 #define GK_DEV_TIMEOUT 2      /* a bounded look-back wait gave up; outputs invalid */
 #define GK_DEV_BAD_SEGMENTS 4 /* seg_offsets not ascending from 0 to d, or seg_k out of range */
+#define GK_DEV_BAD_SAMPLE 8   /* dgck_*: a sampled position outside [0, d) (it was clamped) */
 
 /*
  * What one Gaussian_k run decided (Algorithm 1 of the paper).  For the
@@ -138,6 +139,44 @@ int topk_exact(const float* u, int64_t d, int64_t k, int32_t* idx_out, float* va
  */
 int topk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                   float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
+/*
+ * dgck_select -- DGC_k, the hierarchical sampling selector the paper compares
+ * Gaussian_k with (Section 3.3; Section 4.3 uses a 1 % sample).  The paper says
+ * only that a small random sample estimates the threshold and that top-k
+ * selection runs twice on subsets of the vector; the steps taken here:
+ *   1. tau = the k_m-th largest of { |u[sample_idx[j]]| : j < m },
+ *      k_m = ceil(k * m / d)                       (first top-k, on the sample);
+ *   2. candidates = { i : |u_i| >= tau }, n of them;
+ *   3. n > k: the k largest candidates, ties toward the lower index (second
+ *      top-k, on the candidates); otherwise all n candidates.
+ * min(n, k) pairs are written in ascending index order.
+ *
+ *   u          DEVICE in   d floats, not modified (16-byte aligned)
+ *   sample_idx DEVICE in   m int32 positions in [0, d), repeats allowed: the random
+ *                          draw is the caller's.  A position outside the range is
+ *                          clamped and flagged GK_DEV_BAD_SAMPLE.
+ *   m          sample size, 1 <= m <= 2^31 - 1
+ *   idx_out    DEVICE out  k ints;   val_out  DEVICE out  k floats
+ *   nnz_out    DEVICE out  one int64: min(n, k)
+ * One cooperative kernel; vectors of more than 448 rows of 4096 elements per SM
+ * (271 M elements on 148 SMs) and devices without cooperative launch return
+ * GK_ERR_LIMIT.
+ */
+int dgck_select(const float* u, int64_t d, int64_t k, const int32_t* sample_idx, int64_t m,
+                int32_t* idx_out, float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
+/*
+ * dgck_sparsify -- Eq. 2 of the paper with Comp_k = DGC_k: u = g + eps (the sample
+ * is taken from u), selection as in dgck_select, eps <- u - Comp(u).  g, eps as
+ * for gk_sparsify; the other arguments as for dgck_select.
+ */
+int dgck_sparsify(const float* g, float* eps, int64_t d, int64_t k, const int32_t* sample_idx,
+                  int64_t m, int32_t* idx_out, float* val_out, int64_t* nnz_out, gk_stream_t stream);
+
+/* Synchronise `stream` and write what the last dgck_* call on it decided to HOST
+ * host_out[0..3]: the fp32 bit pattern of tau, n, k_m, pairs written. */
+int dgck_last_info(gk_stream_t stream, int64_t* host_out);
 
 /*
  * gk_sparsify_host -- gk_sparsify for HOST buffers (Eq. 2, Algorithm 1): copies g

@@ -18,12 +18,13 @@ LIB_PATH = os.path.join(HERE, "libgk_b200.so")
 GK_DEV_TRUNCATED = 1
 GK_DEV_TIMEOUT = 2
 GK_DEV_BAD_SEGMENTS = 4
+GK_DEV_BAD_SAMPLE = 8
 
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
-    "gk_error_ratio",
+    "gk_error_ratio", "dgck_select", "dgck_sparsify", "dgck_last_info",
 ]
 
 
@@ -76,6 +77,12 @@ def load() -> C.CDLL:
     L.gk_sparsify_static.restype = C.c_int
     L.gk_error_ratio.argtypes = [vp, i64, vp, vp, vp, C.POINTER(C.c_double)]
     L.gk_error_ratio.restype = C.c_int
+    L.dgck_select.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp]
+    L.dgck_select.restype = C.c_int
+    L.dgck_sparsify.argtypes = [vp, vp, i64, i64, vp, i64, vp, vp, vp, vp]
+    L.dgck_sparsify.restype = C.c_int
+    L.dgck_last_info.argtypes = [vp, C.POINTER(i64)]
+    L.dgck_last_info.restype = C.c_int
     L.gk_sparsify_segmented.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.topk_exact.argtypes = [vp, i64, i64, vp, vp, vp]
     L.topk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
@@ -180,6 +187,30 @@ def topk_sparsify(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
     _check(load().topk_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), g.numel(), k,
                                 _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
                                 _dev(nnz_out, torch.int64), _stream()))
+
+
+def dgck_select(u, k: int, sample_idx, idx_out, val_out, nnz_out) -> None:
+    """DGC_k on a given vector (see gk.h): sampled threshold, then the k largest candidates."""
+    import torch
+    _check(load().dgck_select(_dev(u, torch.float32), u.numel(), k, _dev(sample_idx, torch.int32),
+                              sample_idx.numel(), _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
+                              _dev(nnz_out, torch.int64), _stream()))
+
+
+def dgck_sparsify(g, eps, k: int, sample_idx, idx_out, val_out, nnz_out) -> None:
+    """One error-compensated step with DGC_k as the compressor (see gk.h)."""
+    import torch
+    _check(load().dgck_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), g.numel(), k,
+                                _dev(sample_idx, torch.int32), sample_idx.numel(), _dev(idx_out, torch.int32),
+                                _dev(val_out, torch.float32), _dev(nnz_out, torch.int64), _stream()))
+
+
+def dgck_last_info():
+    """(tau_bits, n_candidates, k_m, pairs_written) of the last dgck_* call on the current
+    stream.  Synchronises the stream."""
+    out = (C.c_int64 * 4)()
+    _check(load().dgck_last_info(_stream(), out))
+    return int(out[0]), int(out[1]), int(out[2]), int(out[3])
 
 
 def gk_sparsify_host(g, eps, k: int, idx_out, val_out):

@@ -63,6 +63,9 @@ struct Ctrl {
     unsigned long long phase_t[8];
     // gk_error_ratio: ratio, ||u - Comp(u)||^2, ||u||^2
     double diag[4];
+    // DGC_k: key of the sampled threshold, candidates at or above it, rank taken in the sample,
+    // pairs written
+    unsigned long long dgc[4];
 };
 
 struct Workspace {

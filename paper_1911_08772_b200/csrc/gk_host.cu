@@ -162,6 +162,17 @@ extern "C" int gk_last_stats(gk_stream_t stream, gk_stats* host_out) {
     return GK_OK;
 }
 
+extern "C" int dgck_last_info(gk_stream_t stream, int64_t* host_out) {
+    if (!host_out) return GK_ERR_NULL;
+    Workspace* ws = find_workspace((cudaStream_t)stream);
+    if (!ws) return GK_ERR_NULL;
+    GK_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    unsigned long long v[4];
+    GK_CUDA_TRY(cudaMemcpy(v, ws->ctrl->dgc, sizeof(v), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 4; ++i) host_out[i] = (int64_t)v[i];
+    return GK_OK;
+}
+
 extern "C" int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* host_out) {
     if (!host_out) return GK_ERR_NULL;
     Workspace* ws = find_workspace((cudaStream_t)stream);

@@ -21,7 +21,7 @@ def declared_functions():
     text = open(os.path.join(ROOT, "include", "gk.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"\b([a-z_0-9]+)\s*\(", text)
-    return sorted({n for n in names if n.startswith(("gk_", "topk_"))})
+    return sorted({n for n in names if n.startswith(("gk_", "topk_", "dgck_"))})
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -84,3 +84,16 @@ def test_binding_refuses_cpu_tensors(lib):
     with pytest.raises(binding.GkError):
         binding.gk_sparsify(t, t.clone(), 1, torch.zeros(8, dtype=torch.int32), t.clone(),
                             torch.zeros(1, dtype=torch.int64))
+
+
+def test_dgck_argument_validation_happens_on_the_host(lib):
+    a = 0x1000
+    st = None
+    assert lib.dgck_select(None, 10, 1, a, 5, a, a, a, st) == -1
+    assert lib.dgck_select(a, 10, 1, None, 5, a, a, a, st) == -1
+    assert lib.dgck_select(a, 0, 1, a, 5, a, a, a, st) == -2
+    assert lib.dgck_select(a, 10, 1, a, 0, a, a, a, st) == -2
+    assert lib.dgck_select(a, 10, 11, a, 5, a, a, a, st) == -3
+    assert lib.dgck_select(a + 4, 10, 1, a, 5, a, a, a, st) == -4
+    assert lib.dgck_sparsify(a, a + 16, 10, 1, a, 5, a, a, a, st) == -5
+    assert lib.dgck_sparsify(a, None, 10, 1, a, 5, a, a, a, st) == -1
