@@ -230,25 +230,28 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         const bool any_neg = cs[0] < 0.f;
         const unsigned short* trow = table + w;
         // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
-        // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows
-        const float4* fp = e4 + first4;  // the row the next fetch brings in
-        auto fetch_u = [&](int r) {
-            if (r < first_kept) cp_async16(gring + ((r & (kRing - 1)) << 10) + tid, fp);
+        // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows.  They are
+        // taken from the last written to the first: the rows written last are the ones most
+        // likely still in L2, and reading them first keeps the misses on the oldest rows from
+        // pushing them out before their turn.
+        int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;  // the row the next fetch brings in
+        auto fetch_u = [&](int q) {   // q-th row in this order: local row first_kept - 1 - q
+            if (q < first_kept) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, e4 + fo);
             cp_async_commit();
-            fp += stride4;
+            fo -= stride4;
         };
         auto row_max = [&](int r) -> unsigned int {
             return any_neg ? always : (unsigned int)trow[r * kFusedWarps];
         };
 #pragma unroll
-        for (int r = 0; r < kRing - 1; ++r) fetch_u(r);
+        for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
         static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
         int r = 0;
 #pragma unroll 2
-        for (; r < first_kept; ++r) {
-            fetch_u(r + kRing - 1);
+        for (int q = 0; q < first_kept; ++q) {
+            fetch_u(q + kRing - 1);
             cp_async_wait<kRing - 1>();
-            count_float4(gring[((r & (kRing - 1)) << 10) + tid], row_max(r), cs, tier, acc);
+            count_float4(gring[((q & (kRing - 1)) << 10) + tid], row_max(first_kept - 1 - q), cs, tier, acc);
         }
         cp_async_wait<0>();
         for (r = first_kept; r < nrows; ++r) {
