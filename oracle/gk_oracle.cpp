@@ -294,4 +294,34 @@ int64_t oracle_dgck_sparsify(const float* g, float* eps, int64_t d, int64_t k, c
     return n;
 }
 
+// ---------------------------------------------------------------------------
+// Eq. 2, the update of the model from the exchanged messages:
+//     x <- x + alpha * sum_p Comp_k(u^p),      alpha = -eta / P in the paper.
+// Rank p's message is the list (idx[p * cap + j], val[p * cap + j]), j < nnz[p]
+// (what the sparsifier wrote).  The sum over the workers is taken in rank
+// order p = 0, 1, ... in fp32, one IEEE addition per term, starting from the
+// first term; then one multiplication by alpha and one addition to x.  Only
+// positions that occur in some message are touched.  The paper does not say
+// in which order the P terms are added; rank order is this repository's choice.
+// ---------------------------------------------------------------------------
+void oracle_apply_sparse(float* x, int64_t d, const int32_t* idx, const float* val, const int64_t* nnz,
+                         int32_t P, int64_t cap, float alpha) {
+    std::vector<float> s((size_t)d, 0.0f);
+    std::vector<unsigned char> seen((size_t)d, 0);
+    for (int32_t p = 0; p < P; ++p) {
+        for (int64_t j = 0; j < nnz[p]; ++j) {
+            const int64_t i = idx[(int64_t)p * cap + j];
+            const float v = val[(int64_t)p * cap + j];
+            if (!seen[(size_t)i]) { s[(size_t)i] = v; seen[(size_t)i] = 1; }
+            else s[(size_t)i] = s[(size_t)i] + v;
+        }
+    }
+    for (int64_t i = 0; i < d; ++i) {
+        if (seen[(size_t)i]) {
+            const float t = alpha * s[(size_t)i];
+            x[i] = x[i] + t;
+        }
+    }
+}
+
 }  // extern "C"

@@ -81,6 +81,8 @@ def lib() -> C.CDLL:
         L.oracle_topk_exact.restype = None
         L.oracle_error_ratio.argtypes = [fp, C.c_int64, ip, C.c_int64]
         L.oracle_error_ratio.restype = C.c_double
+        L.oracle_apply_sparse.argtypes = [fp, C.c_int64, ip, fp, lp, C.c_int32, C.c_int64, C.c_float]
+        L.oracle_apply_sparse.restype = None
         L.oracle_dgck_select.argtypes = [fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
         L.oracle_dgck_select.restype = C.c_int64
         L.oracle_dgck_sparsify.argtypes = [fp, fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
@@ -225,3 +227,14 @@ def dgck_sparsify(g: np.ndarray, eps: np.ndarray, k: int, sample_idx: np.ndarray
     n = lib().oracle_dgck_sparsify(_f(g), _f(eps), d, k, _i(sample_idx), sample_idx.shape[0], _i(idx), _f(val),
                                    _l(info))
     return idx[:n].copy(), val[:n].copy(), DgcInfo(int(info[0]), int(info[1]), int(info[2]))
+
+
+def apply_sparse(x: np.ndarray, idx: np.ndarray, val: np.ndarray, nnz: np.ndarray, cap: int, alpha: float) -> None:
+    """x += alpha * (sum over ranks of their messages), IN PLACE (Eq. 2).  idx, val: P * cap
+    entries, rank p's list at [p * cap, p * cap + nnz[p])."""
+    P = nnz.shape[0]
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    val = np.ascontiguousarray(val, dtype=np.float32)
+    nnz = np.ascontiguousarray(nnz, dtype=np.int64)
+    assert idx.shape[0] == P * cap and val.shape[0] == P * cap
+    lib().oracle_apply_sparse(_f(x), x.shape[0], _i(idx), _f(val), _l(nnz), P, cap, alpha)

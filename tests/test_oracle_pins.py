@@ -517,3 +517,88 @@ def test_dgck_sparsify_identity():
     comp[idx] = val
     assert np.array_equal(bits(comp + eps), bits(u + np.float32(0)))  # Comp(u) + eps_new == u
     assert np.all(eps[idx] == 0) and np.array_equal(bits(np.delete(eps, idx)), bits(np.delete(u, idx)))
+
+
+# --------------------------------------------------------------------------- Eq. 2: the update from P messages
+def _messages(rng, d, P, cap, dense=False):
+    idx = np.zeros(P * cap, dtype=np.int32)
+    val = np.zeros(P * cap, dtype=np.float32)
+    nnz = np.zeros(P, dtype=np.int64)
+    for p in range(P):
+        n = int(rng.integers(0, cap + 1)) if not dense else cap
+        pos = np.sort(rng.choice(d, size=n, replace=False)).astype(np.int32)
+        idx[p * cap:p * cap + n] = pos
+        val[p * cap:p * cap + n] = rng.standard_normal(n).astype(np.float32)
+        nnz[p] = n
+    return idx, val, nnz
+
+
+def test_apply_sparse_single_rank_is_a_scaled_scatter_add():
+    rng = wl.misc_rng(50)
+    d, cap = 5000, 300
+    idx, val, nnz = _messages(rng, d, 1, cap)
+    x = rng.standard_normal(d).astype(np.float32)
+    want = x.copy()
+    n = int(nnz[0])
+    alpha = np.float32(-0.125)
+    want[idx[:n]] = want[idx[:n]] + alpha * val[:n]     # numpy fp32: one multiply, one add
+    orc.apply_sparse(x, idx, val, nnz, cap, float(alpha))
+    assert np.array_equal(bits(x), bits(want))
+
+
+def test_apply_sparse_rank_order_brute_force_and_exact_small_integers():
+    rng = wl.misc_rng(51)
+    d, P, cap = 400, 5, 120          # dense enough for many positions to occur in several ranks
+    idx, val, nnz = _messages(rng, d, P, cap)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    alpha = np.float32(0.3)
+    want = x0.copy()
+    for i in range(d):
+        s, hit = np.float32(0), False
+        for p in range(P):
+            lst = idx[p * cap:p * cap + int(nnz[p])]
+            j = np.nonzero(lst == i)[0]
+            if j.size:
+                v = val[p * cap + int(j[0])]
+                s = v if not hit else np.float32(s + v)
+                hit = True
+        if hit:
+            want[i] = np.float32(want[i] + np.float32(alpha * s))
+    x = x0.copy()
+    orc.apply_sparse(x, idx, val, nnz, cap, float(alpha))
+    assert np.array_equal(bits(x), bits(want))
+    # small integers: every order of additions is exact, so the fp64 scatter-add agrees exactly
+    vi = rng.integers(-8, 9, size=P * cap).astype(np.float32)
+    x = np.zeros(d, dtype=np.float32)
+    orc.apply_sparse(x, idx, vi, nnz, cap, 2.0)
+    ref = np.zeros(d)
+    for p in range(P):
+        n = int(nnz[p])
+        np.add.at(ref, idx[p * cap:p * cap + n], 2.0 * vi[p * cap:p * cap + n].astype(np.float64))
+    assert np.array_equal(x.astype(np.float64), ref)
+    # untouched positions keep their bits (including -0.0)
+    x = np.full(d, -0.0, dtype=np.float32)
+    orc.apply_sparse(x, idx, val, nnz, cap, 1.0)
+    touched = np.zeros(d, dtype=bool)
+    for p in range(P):
+        touched[idx[p * cap:p * cap + int(nnz[p])]] = True
+    assert np.all(bits(x[~touched]) == 0x80000000)
+
+
+def test_apply_sparse_sums_what_the_workers_selected():
+    # P workers sparsify their own vectors; the update applied to x = 0 with alpha = 1 equals
+    # the sum of their dense Comp_k(u^p) vectors (fp64 reference, fp32 rounding tolerance)
+    rng = wl.misc_rng(52)
+    d, P, k = 50_000, 4, 500
+    cap = 2 * k
+    idx = np.zeros(P * cap, dtype=np.int32); val = np.zeros(P * cap, dtype=np.float32)
+    nnz = np.zeros(P, dtype=np.int64)
+    dense = np.zeros(d)
+    for p in range(P):
+        u = (rng.standard_normal(d) * 1e-2).astype(np.float32)
+        ti, tv = orc.topk_exact(u, k)
+        idx[p * cap:p * cap + k] = ti; val[p * cap:p * cap + k] = tv; nnz[p] = k
+        dense[ti] += tv.astype(np.float64)
+    x = np.zeros(d, dtype=np.float32)
+    orc.apply_sparse(x, idx, val, nnz, cap, 1.0)
+    assert np.allclose(x, dense, rtol=1e-6, atol=1e-9)
