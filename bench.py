@@ -435,6 +435,31 @@ def run_ours(args):
                     "cleared slot)"}
     del eps2, us, smps
 
+    # ---- the model update of Eq. 2 from P workers' messages (P workers emulated one after the
+    # other on this GPU, each with its own gradient; messages = exact Top_k lists of k pairs)
+    upd = {}
+    x_model = torch.zeros(d, dtype=torch.float32, device=dev)
+    eps4 = torch.zeros_like(epss[0])
+    for P_w in (8, 16):
+        m_idx = torch.empty(P_w * k, dtype=torch.int32, device=dev)
+        m_val = torch.empty(P_w * k, dtype=torch.float32, device=dev)
+        m_nnz = torch.zeros(P_w, dtype=torch.int64, device=dev)
+        for p_w in range(P_w):
+            eps4.zero_()
+            gk.topk_sparsify(gs[p_w % n_rot], eps4, k, m_idx[p_w * k:(p_w + 1) * k], m_val[p_w * k:(p_w + 1) * k],
+                             m_nnz[p_w:p_w + 1])
+        for t in range(3):
+            gk.gk_apply_gathered(x_model, m_idx, m_val, m_nnz, k, -0.01 / P_w)
+        ms_up = time_region(torch, lambda t: gk.gk_apply_gathered(x_model, m_idx, m_val, m_nnz, k, -0.01 / P_w),
+                            Kt) / Kt
+        upd[f"P={P_w}"] = {"ms": ms_up, "entries": P_w * k,
+                           "entries_per_s": P_w * k / (ms_up * 1e-3),
+                           "list_gbs_8B_per_entry": 8.0 * P_w * k / ms_up / 1e6}
+        del m_idx, m_val, m_nnz
+    upd["note"] = ("gk_apply_gathered: x += alpha * sum_p Comp_k(u^p), rank order, one kernel; messages resident "
+                   "(no all-gather in this number)")
+    del x_model, eps4
+
     # ---- the error ratio of Eq. 5 for one Gaussian_k step and one Top_k step from eps = 0
     diag = {"bound_eq4_1_minus_k_over_d": 1.0 - k / d, "bound_theorem1_squared": (1.0 - k / d) ** 2}
     eps3 = torch.zeros_like(epss[0])
@@ -502,7 +527,7 @@ def run_ours(args):
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
                  "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
-        "dgck": dgck, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
+        "dgck": dgck, "update_from_messages": upd, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
         "clocks": sampler.summary(),
     }
     print(json.dumps(line))

@@ -50,6 +50,7 @@ typedef enum gk_status {
 #define GK_DEV_TIMEOUT 2      /* a bounded look-back wait gave up; outputs invalid */
 #define GK_DEV_BAD_SEGMENTS 4 /* seg_offsets not ascending from 0 to d, or seg_k out of range */
 #define GK_DEV_BAD_SAMPLE 8   /* dgck_*: a sampled position outside [0, d) (it was clamped) */
+#define GK_DEV_BAD_INDEX 16   /* gk_apply_*: a message index outside [0, d) (the entry was skipped) */
 
 /*
  * What one Gaussian_k run decided (Algorithm 1 of the paper).  For the
@@ -177,6 +178,33 @@ int dgck_sparsify(const float* g, float* eps, int64_t d, int64_t k, const int32_
 /* Synchronise `stream` and write what the last dgck_* call on it decided to HOST
  * host_out[0..3]: the fp32 bit pattern of tau, n, k_m, pairs written. */
 int dgck_last_info(gk_stream_t stream, int64_t* host_out);
+
+/*
+ * gk_apply_sparse -- the model update of Eq. 2 from the P workers' messages:
+ *     x <- x + alpha * sum_p Comp_k(u^p)          (alpha = -eta / P in the paper).
+ * Message p is the ascending (index, value) list a sparsifier call wrote.  The
+ * terms of a position are added in rank order p = 0, 1, ... in fp32 (one
+ * addition per term), the sum is multiplied by alpha and added to x; positions
+ * that occur in no message are not touched.  The paper does not fix the order
+ * of the P terms; rank order makes the result independent of timing.
+ *
+ *   x          DEVICE i/o  d floats
+ *   idx_lists  HOST   in   P pointers to DEVICE int32 lists, each strictly ascending;
+ *   val_lists  HOST   in   P pointers to DEVICE float lists.  A list may live in
+ *                          another GPU's memory that this device can address (peer
+ *                          access): the kernel reads the lists with plain loads.
+ *   nnz        DEVICE in   P int64: entries of each list (values above cap count as cap)
+ *   P          number of messages, 1 <= P <= 64;  cap: upper bound of every nnz[p]
+ * One kernel, no scratch vector, no atomics on x.  An index outside [0, d) is
+ * skipped and flagged GK_DEV_BAD_INDEX in the status word gk_last_stats returns.
+ *
+ * gk_apply_gathered -- the same for messages in one buffer (as an all-gather
+ * leaves them): list p starts at idx + p * cap and val + p * cap (DEVICE).
+ */
+int gk_apply_sparse(float* x, int64_t d, const int32_t* const* idx_lists, const float* const* val_lists,
+                    const int64_t* nnz, int32_t P, int64_t cap, float alpha, gk_stream_t stream);
+int gk_apply_gathered(float* x, int64_t d, const int32_t* idx, const float* val, const int64_t* nnz,
+                      int32_t P, int64_t cap, float alpha, gk_stream_t stream);
 
 /*
  * gk_sparsify_host -- gk_sparsify for HOST buffers (Eq. 2, Algorithm 1): copies g

@@ -19,12 +19,14 @@ GK_DEV_TRUNCATED = 1
 GK_DEV_TIMEOUT = 2
 GK_DEV_BAD_SEGMENTS = 4
 GK_DEV_BAD_SAMPLE = 8
+GK_DEV_BAD_INDEX = 16
 
 EXPORTS = [
     "gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
     "gk_error_ratio", "dgck_select", "dgck_sparsify", "dgck_last_info",
+    "gk_apply_sparse", "gk_apply_gathered",
 ]
 
 
@@ -77,6 +79,10 @@ def load() -> C.CDLL:
     L.gk_sparsify_static.restype = C.c_int
     L.gk_error_ratio.argtypes = [vp, i64, vp, vp, vp, C.POINTER(C.c_double)]
     L.gk_error_ratio.restype = C.c_int
+    L.gk_apply_sparse.argtypes = [vp, i64, C.POINTER(vp), C.POINTER(vp), vp, i32, i64, C.c_float, vp]
+    L.gk_apply_sparse.restype = C.c_int
+    L.gk_apply_gathered.argtypes = [vp, i64, vp, vp, vp, i32, i64, C.c_float, vp]
+    L.gk_apply_gathered.restype = C.c_int
     L.dgck_select.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp]
     L.dgck_select.restype = C.c_int
     L.dgck_sparsify.argtypes = [vp, vp, i64, i64, vp, i64, vp, vp, vp, vp]
@@ -211,6 +217,27 @@ def dgck_last_info():
     out = (C.c_int64 * 4)()
     _check(load().dgck_last_info(_stream(), out))
     return int(out[0]), int(out[1]), int(out[2]), int(out[3])
+
+
+def gk_apply_gathered(x, idx, val, nnz, cap: int, alpha: float) -> None:
+    """x += alpha * (sum over the P = nnz.numel() messages), list p at [p * cap, p * cap + nnz[p])
+    of idx / val (Eq. 2; see gk.h)."""
+    import torch
+    P = nnz.numel()
+    if idx.numel() < P * cap or val.numel() < P * cap:
+        raise GkError("idx / val hold fewer than P * cap entries")
+    _check(load().gk_apply_gathered(_dev(x, torch.float32), x.numel(), _dev(idx, torch.int32),
+                                    _dev(val, torch.float32), _dev(nnz, torch.int64), P, cap, alpha, _stream()))
+
+
+def gk_apply_sparse(x, idx_lists, val_lists, nnz, cap: int, alpha: float) -> None:
+    """The same with one tensor per message (each may live in a peer GPU's memory)."""
+    import torch
+    P = len(idx_lists)
+    ip = (C.c_void_p * P)(*[_dev(t, torch.int32) for t in idx_lists])
+    vp_ = (C.c_void_p * P)(*[_dev(t, torch.float32) for t in val_lists])
+    _check(load().gk_apply_sparse(_dev(x, torch.float32), x.numel(), ip, vp_, _dev(nnz, torch.int64), P, cap,
+                                  alpha, _stream()))
 
 
 def gk_sparsify_host(g, eps, k: int, idx_out, val_out):
