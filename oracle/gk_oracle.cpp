@@ -324,4 +324,26 @@ void oracle_apply_sparse(float* x, int64_t d, const int32_t* idx, const float* v
     }
 }
 
+// ---------------------------------------------------------------------------
+// The histogram of u that the paper's gradient-distribution figures show
+// (Section 3.1, Fig. 2, and the cumulative curves of the appendix): nbins equal bins
+// over [lo, hi), plus one count below and one above.  Floating point decides
+// an integer here, so the rule is fixed in fp32, the vector's own precision:
+//     t = (u_i - lo) * inv_w    (one fp32 subtraction, one fp32 multiplication,
+//                                inv_w = nbins / (hi - lo) given by the caller)
+//     bin = floor(t);  t < 0 -> "below";  t >= nbins (or NaN) -> "above".
+// counts: nbins + 2 entries: [0] below, [1 .. nbins] the bins, [nbins + 1] above.
+// The cumulative distribution is the running sum of these counts over d.
+// ---------------------------------------------------------------------------
+void oracle_histogram(const float* u, int64_t d, float lo, float inv_w, int32_t nbins, int64_t* counts) {
+    for (int32_t b = 0; b < nbins + 2; ++b) counts[b] = 0;
+    for (int64_t i = 0; i < d; ++i) {
+        const float diff = u[i] - lo;
+        const float t = diff * inv_w;
+        if (t < 0.0f) counts[0] += 1;
+        else if (!(t < (float)nbins)) counts[nbins + 1] += 1;
+        else counts[1 + (int32_t)std::floor(t)] += 1;
+    }
+}
+
 }  // extern "C"

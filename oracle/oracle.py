@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
         L.oracle_error_ratio.restype = C.c_double
         L.oracle_apply_sparse.argtypes = [fp, C.c_int64, ip, fp, lp, C.c_int32, C.c_int64, C.c_float]
         L.oracle_apply_sparse.restype = None
+        L.oracle_histogram.argtypes = [fp, C.c_int64, C.c_float, C.c_float, C.c_int32, lp]
+        L.oracle_histogram.restype = None
         L.oracle_dgck_select.argtypes = [fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
         L.oracle_dgck_select.restype = C.c_int64
         L.oracle_dgck_sparsify.argtypes = [fp, fp, C.c_int64, C.c_int64, ip, C.c_int64, ip, fp, lp]
@@ -238,3 +240,10 @@ def apply_sparse(x: np.ndarray, idx: np.ndarray, val: np.ndarray, nnz: np.ndarra
     nnz = np.ascontiguousarray(nnz, dtype=np.int64)
     assert idx.shape[0] == P * cap and val.shape[0] == P * cap
     lib().oracle_apply_sparse(_f(x), x.shape[0], _i(idx), _f(val), _l(nnz), P, cap, alpha)
+
+
+def histogram(u: np.ndarray, lo: float, inv_w: float, nbins: int) -> np.ndarray:
+    """Counts of u in nbins equal bins from lo (bin width 1 / inv_w): [below, bins..., above]."""
+    counts = np.zeros(nbins + 2, dtype=np.int64)
+    lib().oracle_histogram(_f(u), u.shape[0], lo, inv_w, nbins, _l(counts))
+    return counts

@@ -602,3 +602,40 @@ def test_apply_sparse_sums_what_the_workers_selected():
     x = np.zeros(d, dtype=np.float32)
     orc.apply_sparse(x, idx, val, nnz, cap, 1.0)
     assert np.allclose(x, dense, rtol=1e-6, atol=1e-9)
+
+
+# --------------------------------------------------------------------------- histogram of u (Section 3.1, Fig. 2)
+def test_histogram_on_a_dyadic_grid_equals_numpy():
+    # values on a grid of 2^-10 with dyadic bin edges: every fp32 operation of the rule is
+    # exact, so numpy's fp64 histogram must agree count for count
+    rng = wl.misc_rng(60)
+    u = (rng.integers(-3000, 3000, size=200_000) / 1024.0).astype(np.float32)
+    lo, hi, nbins = -2.0, 2.0, 64
+    counts = orc.histogram(u, lo, nbins / (hi - lo), nbins)
+    ref, _ = np.histogram(u.astype(np.float64), bins=nbins, range=(lo, hi))
+    # numpy puts x == hi into the last bin; the rule here counts it as "above"
+    at_hi = int((u == hi).sum())
+    ref[-1] -= at_hi
+    assert np.array_equal(counts[1:-1], ref)
+    assert counts[0] == int((u < lo).sum()) and counts[-1] == int((u >= hi).sum())
+    assert counts.sum() == u.size
+
+
+def test_histogram_hand_case_and_edges():
+    u = np.array([-1.0, -0.5, -0.0, 0.0, 0.25, 0.4999, 0.5, 0.75, 1.0, 7.0, -7.0], dtype=np.float32)
+    counts = orc.histogram(u, -1.0, 2.0, 4)   # bins [-1,-.5) [-.5,0) [0,.5) [.5,1)
+    assert counts.tolist() == [1, 1, 1, 4, 2, 2]
+    assert orc.histogram(np.array([np.nan], dtype=np.float32), 0.0, 1.0, 3).tolist() == [0, 0, 0, 0, 1]
+
+
+def test_histogram_cdf_of_gaussian_input_matches_the_normal_cdf():
+    d = 1 << 21
+    u = wl.normal(d, 1e-3, step=9)
+    nbins, lo, hi = 200, -5e-3, 5e-3
+    counts = orc.histogram(u, np.float32(lo), np.float32(nbins / (hi - lo)), nbins)
+    cdf = np.cumsum(counts)[:-1] / d                      # P(u < edge_j), j = 0 .. nbins
+    edges = np.linspace(lo, hi, nbins + 1)
+    assert np.max(np.abs(cdf - sps.norm.cdf(edges / 1e-3))) < 5.0 / math.sqrt(d)
+    # against numpy on the same data: only values within rounding of an edge may move
+    ref, _ = np.histogram(u.astype(np.float64), bins=nbins, range=(lo, hi))
+    assert np.abs(counts[1:-1] - ref).sum() <= 1e-5 * d
