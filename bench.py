@@ -474,7 +474,16 @@ def run_ours(args):
         gk.gk_stage_timing(False)
         diag[name] = {"error_ratio": r[0], "nnz": int(nnz.item()), "ms": acc / 10,
                       "gbs_4B_per_elem": 4.0 * d / (acc / 10) / 1e6}
-    del eps3
+    # the histogram of u (Section 3.1): 512 bins over +-4 sigma of one step's u (eps3 holds it, minus
+    # the selected entries)
+    hcnt = torch.zeros(514, dtype=torch.int64, device=dev)
+    sig = float(eps3[:1_000_000].std().item()) or 1.0
+    for _ in range(3):
+        gk.gk_histogram(eps3, -4 * sig, 512 / (8 * sig), hcnt)
+    ms_h = time_region(torch, lambda t: gk.gk_histogram(eps3, -4 * sig, 512 / (8 * sig), hcnt), 20) / 20
+    diag["histogram"] = {"bins": 512, "ms": ms_h, "gbs_4B_per_elem": 4.0 * d / ms_h / 1e6,
+                         "inside": int(hcnt[1:-1].sum().item()), "outside": int(hcnt[0].item() + hcnt[-1].item())}
+    del eps3, hcnt
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
     hg = [torch.from_numpy(w.grad(j, None)).pin_memory() for j in range(2)]

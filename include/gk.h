@@ -234,6 +234,23 @@ int gk_error_ratio(const float* eps, int64_t d, const float* val, const int64_t*
                    gk_stream_t stream, double* host_out);
 
 /*
+ * gk_histogram -- the histogram of u shown in the paper's gradient-distribution
+ * figures (Section 3.1, Fig. 2; its running sum over d is the cumulative curve
+ * of the appendix).  nbins equal bins starting at lo, bin width 1 / inv_w:
+ *     t = (u_i - lo) * inv_w in fp32 (one subtraction, one multiplication);
+ *     t < 0 counts as "below", t >= nbins (or NaN) as "above", else bin floor(t).
+ *
+ *   u          DEVICE in   d floats (16-byte aligned), not modified
+ *   lo, inv_w  lower edge of the first bin; inv_w = nbins / (hi - lo) > 0, as a float
+ *   nbins      1 <= nbins <= 8192
+ *   counts_out DEVICE out  nbins + 2 int64: [0] below, [1 .. nbins] the bins,
+ *                          [nbins + 1] above (zeroed by the call)
+ * One pass over u, enqueued on `stream`; does not synchronise.
+ */
+int gk_histogram(const float* u, int64_t d, float lo, float inv_w, int32_t nbins, int64_t* counts_out,
+                 gk_stream_t stream);
+
+/*
  * gk_sparsify_static -- gk_sparsify for callers that must not allocate device
  * memory (the paper has no counterpart: this is a deployment variant of the
  * same step, not another method).  Think of a step that runs under a framework

@@ -26,7 +26,7 @@ EXPORTS = [
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
     "gk_error_ratio", "dgck_select", "dgck_sparsify", "dgck_last_info",
-    "gk_apply_sparse", "gk_apply_gathered",
+    "gk_apply_sparse", "gk_apply_gathered", "gk_histogram",
 ]
 
 
@@ -83,6 +83,8 @@ def load() -> C.CDLL:
     L.gk_apply_sparse.restype = C.c_int
     L.gk_apply_gathered.argtypes = [vp, i64, vp, vp, vp, i32, i64, C.c_float, vp]
     L.gk_apply_gathered.restype = C.c_int
+    L.gk_histogram.argtypes = [vp, i64, C.c_float, C.c_float, i32, vp, vp]
+    L.gk_histogram.restype = C.c_int
     L.dgck_select.argtypes = [vp, i64, i64, vp, i64, vp, vp, vp, vp]
     L.dgck_select.restype = C.c_int
     L.dgck_sparsify.argtypes = [vp, vp, i64, i64, vp, i64, vp, vp, vp, vp]
@@ -238,6 +240,14 @@ def gk_apply_sparse(x, idx_lists, val_lists, nnz, cap: int, alpha: float) -> Non
     vp_ = (C.c_void_p * P)(*[_dev(t, torch.float32) for t in val_lists])
     _check(load().gk_apply_sparse(_dev(x, torch.float32), x.numel(), ip, vp_, _dev(nnz, torch.int64), P, cap,
                                   alpha, _stream()))
+
+
+def gk_histogram(u, lo: float, inv_w: float, counts_out) -> None:
+    """Histogram of u over nbins = counts_out.numel() - 2 equal bins from lo (width 1 / inv_w);
+    counts_out (int64): [below, bins..., above] (see gk.h).  Enqueued on the current stream."""
+    import torch
+    _check(load().gk_histogram(_dev(u, torch.float32), u.numel(), lo, inv_w, counts_out.numel() - 2,
+                               _dev(counts_out, torch.int64), _stream()))
 
 
 def gk_sparsify_host(g, eps, k: int, idx_out, val_out):
