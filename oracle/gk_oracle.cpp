@@ -243,11 +243,11 @@ double oracle_error_ratio(const float* u, int64_t d, const int32_t* idx, int64_t
 }
 
 // ---------------------------------------------------------------------------
-// DGC_k, the hierarchical sampling selector the paper compares against
-// (Section 3.3: "sample only 0.1% to 1% of the gradients to estimate the
-// threshold hierarchically", with two top-k selections on subsets of the
-// vector; Section 4.3: a 1% sample).  The paper gives no more than that; the
-// reading taken here:
+// DGC_k, the hierarchical sampling selector the paper compares against.
+// Section 3.3 describes it in one sentence: a sample of 0.1 % to 1 % of the
+// entries estimates the threshold, and top-k selection runs twice, each time on
+// a subset of the vector; Section 4.3 takes a 1 % sample.  The paper gives no
+// more than that; the reading taken here:
 //   1. the sample is the multiset { |u[s_j]| : j < m } at the positions s_j the
 //      caller drew (the random draw is an input, not part of the arithmetic);
 //   2. first top-k, on the sample: with k_m = ceil(k * m / d) (the density k/d
