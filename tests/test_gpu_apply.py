@@ -109,3 +109,36 @@ def test_apply_after_real_sparsifier_steps(P):
     gk.gk_apply_gathered(dx, didx, dval, dnnz, cap, -0.1 / P)
     assert np.array_equal(bits(dx.cpu().numpy()), bits(want))
     assert int((want != x0).sum()) > 0
+
+
+def test_exchange_and_apply_through_nccl_with_one_rank():
+    """The wrapper end to end on the GPU: a one-rank NCCL group (this box has one GPU), the
+    all-gather of the message, the update kernel; against the oracle."""
+    import os
+    import socket
+    import torch.distributed as dist
+    from paper_1911_08772_b200 import exchange
+
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(DEV))
+    try:
+        rng = wl.misc_rng(4400)
+        d, cap = 200_000, 3000
+        idx, val, nnz = messages(rng, d, 1, cap, 0.7)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        want = x0.copy()
+        orc.apply_sparse(want, idx, val, nnz, cap, -0.05)
+        dx = torch.from_numpy(x0).to(DEV)
+        # buffers longer than cap, as a sparsifier's output buffers are
+        di = torch.cat([torch.from_numpy(idx), torch.full((100,), -3, dtype=torch.int32)]).to(DEV)
+        dv = torch.cat([torch.from_numpy(val), torch.zeros(100)]).to(DEV)
+        exchange.exchange_and_apply(dx, di, dv, torch.from_numpy(nnz).to(DEV), cap, -0.05)
+        torch.cuda.synchronize()
+        assert np.array_equal(bits(dx.cpu().numpy()), bits(want))
+    finally:
+        dist.destroy_process_group()
