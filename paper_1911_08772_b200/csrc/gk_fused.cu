@@ -51,6 +51,9 @@ constexpr int kRing = 8;                               // ring slots; phase B ha
 constexpr int kGroupRows = 8;                          // rows a warp gathers per batch in phase C
 constexpr int kFusedMaxGrid = kFusedGridCap;
 constexpr int kTraceSlots = 8;                         // timestamps per CTA in the optional trace
+// phase C keeps the places of a CTA's survivors (row, warp, lane, element, rank within the
+// segment: one word each) in the ring's shared memory between counting and write-out
+constexpr int kStageCap = kRing * kRowF4 * 4;
 
 struct __align__(128) FusedShared {
     double2 red[kFusedWarps];
@@ -67,6 +70,7 @@ struct __align__(128) FusedShared {
     unsigned int roundtot[kTableMaxRows];  // survivors in each round of rows (G consecutive rows)
     unsigned int rowpre[kTableMaxRows];    // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
+    unsigned int n_staged;                 // survivors put aside in phase C
 };
 
 static_assert((sizeof(FusedShared) + 1023) / 1024 * 1024 + kFusedSmemBudget <= 232448,
@@ -302,6 +306,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
             sh.chosen = alg1_resolve(st, k);
+            sh.n_staged = 0u;
         }
         __syncthreads();
         if (c == 0 && tid == 0) {
@@ -359,38 +364,96 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         auto load_row = [&](int r, int64_t i) -> float4 {
             return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
         };
+        // When this CTA's survivors fit the ring's shared memory (free since phase B), their
+        // places -- row, warp, lane, element, rank within the segment: one word -- are put aside
+        // while they are counted, and the write-out is one thread per survivor instead of one
+        // warp per segment; with many survivors the per-segment work of 32 warps was what the
+        // phase cost.
+        const bool staged = mine <= (unsigned)kStageCap;
+        unsigned int* st_tag = reinterpret_cast<unsigned int*>(gring);
         if (mine != 0u) {
             // step 1: every warp counts the survivors of its qualifying segments; the table
             // entry of a segment is replaced by that count (0 where it cannot qualify).
-            // Qualifying rows are gathered eight at a time so that their loads overlap.
+            int pending = 0;
             for (int r = lane; r < nrows; r += 32) {
                 const bool ql = all_pass || table[r * kFusedWarps + w] > thr16;
                 table[r * kFusedWarps + w] = ql ? kPending : (unsigned short)0;
+                pending += ql;
             }
+            pending = __reduce_add_sync(0xffffffffu, pending);
             __syncwarp();
-            for (int cursor = 0; cursor < nrows;) {
-                const int n = gather(cursor, true);
-                float4 v[kGroupRows];
+            const unsigned int lanes_below = (1u << lane) - 1u;
+            // one segment: x is this thread's float4 of local row r, i its float4 index
+            auto count_cell = [&](const int r, const float4 x, const int64_t i) {
+                const unsigned int m = i < n4 ? mask_above(x, thr) : 0u;
+                const unsigned int cnt = __reduce_add_sync(0xffffffffu, __popc(m));
+                if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
+                if (staged && cnt != 0u) {
+                    unsigned int base = 0u;
+                    if (lane == 0) base = atomicAdd(&sh.n_staged, cnt);
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    unsigned int rank = 0u;
+                    if (cnt > 1u) {
+                        // one ballot per element of the float4: the bits below this lane are its rank
+                        const unsigned int b0 = __ballot_sync(0xffffffffu, m & 1u), b1 = __ballot_sync(0xffffffffu, m & 2u),
+                                           b2 = __ballot_sync(0xffffffffu, m & 4u), b3 = __ballot_sync(0xffffffffu, m & 8u);
+                        rank = __popc(b0 & lanes_below) + __popc(b1 & lanes_below) + __popc(b2 & lanes_below) +
+                               __popc(b3 & lanes_below);
+                    }
+                    if (m) {
+                        const unsigned int place = ((unsigned int)r << 19) | ((unsigned int)w << 14) | ((unsigned int)lane << 9);
 #pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (q < n) {
-                        const int r = sh.qrow[w][q];
-                        const int64_t i = (first4 + (int64_t)r * stride4);
-                        if (i < n4) v[q] = load_row(r, i);
+                        for (int t = 0; t < 4; ++t) {
+                            if (m & (1u << t)) {
+                                st_tag[base + rank] = place | ((unsigned int)t << 7) | rank;
+                                ++rank;
+                            }
+                        }
                     }
                 }
+            };
+            if (pending * 4 > nrows) {
+                // many qualifying segments: the rows are taken eight at a time as they come
+                for (int r0 = 0; r0 < nrows; r0 += kGroupRows) {
+                    float4 v[kGroupRows];
+                    bool on[kGroupRows];
 #pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    if (q < n) {
-                        const int r = sh.qrow[w][q];
-                        const int64_t i = (first4 + (int64_t)r * stride4);
-                        const unsigned int cnt =
-                            __reduce_add_sync(0xffffffffu, i < n4 ? __popc(mask_above(v[q], thr)) : 0u);
-                        if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
+                    for (int q = 0; q < kGroupRows; ++q) {
+                        const int r = r0 + q;
+                        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        on[q] = r < nrows && table[r * kFusedWarps + w] == kPending;
+                        if (on[q]) {
+                            const int64_t i = (first4 + (int64_t)r * stride4);
+                            if (i < n4) v[q] = load_row(r, i);
+                        }
                     }
+#pragma unroll
+                    for (int q = 0; q < kGroupRows; ++q)
+                        if (on[q]) count_cell(r0 + q, v[q], first4 + (int64_t)(r0 + q) * stride4);
                 }
-                __syncwarp();
+            } else {
+                // few qualifying segments: they are gathered eight at a time so that their loads overlap
+                for (int cursor = 0; cursor < nrows;) {
+                    const int n = gather(cursor, true);
+                    float4 v[kGroupRows];
+#pragma unroll
+                    for (int q = 0; q < kGroupRows; ++q) {
+                        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (q < n) {
+                            const int r = sh.qrow[w][q];
+                            const int64_t i = (first4 + (int64_t)r * stride4);
+                            if (i < n4) v[q] = load_row(r, i);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < kGroupRows; ++q) {
+                        if (q < n) {
+                            const int r = sh.qrow[w][q];
+                            count_cell(r, v[q], first4 + (int64_t)r * stride4);
+                        }
+                    }
+                    __syncwarp();
+                }
             }
         }
         __syncthreads();
@@ -399,12 +462,25 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         if (tid < nrows) {
             unsigned int mine_row = 0u;
             if (mine != 0u) {
-                const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
+                uint4* tv = reinterpret_cast<uint4*>(table + (size_t)tid * kFusedWarps);
 #pragma unroll
                 for (int q = 0; q < kTableRowBytes / 16; ++q) {
                     const uint4 x = tv[q];
-                    mine_row += (x.x & 0xffffu) + (x.x >> 16) + (x.y & 0xffffu) + (x.y >> 16) +
-                                (x.z & 0xffffu) + (x.z >> 16) + (x.w & 0xffffu) + (x.w >> 16);
+                    if (staged) {
+                        // the entries become the survivors of the row in the warps before each one
+                        // (at most 3968: sixteen bits hold it), which is what the write-out needs
+                        unsigned int ws[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const unsigned int lo = ws[j] & 0xffffu, hi = ws[j] >> 16;
+                            ws[j] = mine_row | ((mine_row + lo) << 16);
+                            mine_row += lo + hi;
+                        }
+                        tv[q] = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+                    } else {
+                        mine_row += (x.x & 0xffffu) + (x.x >> 16) + (x.y & 0xffffu) + (x.y >> 16) +
+                                    (x.z & 0xffffu) + (x.z >> 16) + (x.w & 0xffffu) + (x.w >> 16);
+                    }
                 }
             }
             rowcnt[c + tid * G] = mine_row;
@@ -454,6 +530,27 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 if (tid < nrows) sh.rowpre[tid] += wpre + s - mine_round;
                 __syncthreads();
             }
+            if (staged) {
+                // step 3: one thread per survivor put aside: its place gives its index, where its
+                // value is, and its position in the output
+                const unsigned int n_st = sh.n_staged;
+                for (unsigned int j = tid; j < n_st; j += kFusedThreads) {
+                    const unsigned int tag = st_tag[j];
+                    const unsigned int r = tag >> 19, cell = (tag >> 14) & 31u, ln = (tag >> 9) & 31u, t = (tag >> 7) & 3u,
+                                       rank = tag & 127u;
+                    const long long p = (long long)sh.rowpre[r] + table[r * kFusedWarps + cell] + rank;
+                    if (p < cap) {
+                        const unsigned int in_row = ((cell << 5) | ln) << 2 | t;   // element within the row
+                        const int64_t at = (((int64_t)c + (int64_t)r * G) << 12) + in_row;
+                        const float x = ((int)r >= first_kept)
+                                            ? reinterpret_cast<const float*>(uslot + (size_t)(r % u_slots) * kRowF4)[in_row]
+                                            : __ldcg(eps + at);
+                        idx_out[p] = (int32_t)at;
+                        val_out[p] = x;
+                        eps[at] = 0.0f;
+                    }
+                }
+            } else
             // step 3: every warp writes the survivors of its segments that have any
             for (int cursor = 0; cursor < nrows;) {
                 const int n = gather(cursor, false);
