@@ -41,6 +41,9 @@ constexpr int kSfStages = 4;                           // phase A: rows of g and
 constexpr int kSfRing = 8;                             // ring slots; phase B has kSfRing - 1 rows in flight
 constexpr int kSfGroupRows = 8;
 constexpr unsigned short kSfPending = 0xffffu;
+// phase C keeps the places of a run's survivors (row, warp, lane, element, rank within the
+// 128-element segment: one word each) in the ring's shared memory between counting and write-out
+constexpr int kSfStageCap = kSfRing * kFusedThreads * 4;
 constexpr int kSfLocal = 8;                           // segments of a run whose partial results wait in shared memory
 
 struct __align__(128) SegFusedShared {
@@ -57,6 +60,7 @@ struct __align__(128) SegFusedShared {
     unsigned int rowpre[kSfTableMaxRows];              // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kSfGroupRows];
     unsigned long long total;                          // survivors in the runs before this one
+    unsigned int n_staged;                             // survivors whose places were put aside in phase C
     int ok;
 };
 constexpr int kSfSmemBudget = (232448 - (int)((sizeof(SegFusedShared) + 1023) / 1024 * 1024));
@@ -602,6 +606,8 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
     }
 
     // ------------------------------------------------------------------ phase C
+    if (tid == 0) sh.n_staged = 0u;
+    __syncthreads();
     {
         // threshold of element e, given a segment sx at or before its own (empty segments skipped)
         auto thr_at = [&](int& sx, int64_t e) -> float {
@@ -672,6 +678,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         // step 1: survivors of every qualifying segment into the table (rows come in ascending
         // order, so the warp's position among the segments only moves forward)
         int su1 = s_run;
+        unsigned int* st_tag = reinterpret_cast<unsigned int*>(gring);
         for (int cursor = 0; cursor < nrows;) {
             const int n = gather(cursor, true);
             float4 x[kSfGroupRows];
@@ -691,24 +698,62 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
                     // every lane starts its walk at the segment of the warp's first element
                     const int su = su1 = seg_advance(sh.off, S_use, su1, ((lo4 + (int64_t)r * kRowF4) << 2) + 128 * w);
-                    const unsigned int cnt =
-                        __reduce_add_sync(0xffffffffu, i < hi4 ? __popc(mask_of(x[q], i << 2, su)) : 0u);
+                    const unsigned int m = i < hi4 ? mask_of(x[q], i << 2, su) : 0u;
+                    const unsigned int cnt = __reduce_add_sync(0xffffffffu, __popc(m));
                     if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
+                    if (cnt != 0u) {
+                        // the survivors' places are put aside for the write-out (as long as they fit)
+                        unsigned int base = 0u;
+                        if (lane == 0) base = atomicAdd(&sh.n_staged, cnt);
+                        base = __shfl_sync(0xffffffffu, base, 0);
+                        unsigned int rank = 0u;
+                        if (cnt > 1u) {
+                            const unsigned int b0 = __ballot_sync(0xffffffffu, m & 1u), b1 = __ballot_sync(0xffffffffu, m & 2u),
+                                               b2 = __ballot_sync(0xffffffffu, m & 4u), b3 = __ballot_sync(0xffffffffu, m & 8u);
+                            const unsigned int below = (1u << lane) - 1u;
+                            rank = __popc(b0 & below) + __popc(b1 & below) + __popc(b2 & below) + __popc(b3 & below);
+                        }
+                        if (m && base + cnt <= (unsigned)kSfStageCap) {
+                            const unsigned int place = ((unsigned int)r << 19) | ((unsigned int)w << 14) | ((unsigned int)lane << 9);
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                if (m & (1u << t)) {
+                                    st_tag[base + rank] = place | ((unsigned int)t << 7) | rank;
+                                    ++rank;
+                                }
+                            }
+                        }
+                    }
                 }
             }
             __syncwarp();
         }
         __syncthreads();
+        // all places kept: the write-out is one thread per survivor; else one warp per segment
+        const bool staged = sh.n_staged <= (unsigned)kSfStageCap;
         // step 2: survivors per row (thread t takes row t), a scan over this run's rows, and the
         // run's total to this CTA's word in global memory
         unsigned int mine_row = 0u;
         if (tid < nrows) {
-            const uint4* tv = reinterpret_cast<const uint4*>(table + (size_t)tid * kFusedWarps);
+            uint4* tv = reinterpret_cast<uint4*>(table + (size_t)tid * kFusedWarps);
 #pragma unroll
             for (int q = 0; q < kSfTableRowBytes / 16; ++q) {
                 const uint4 y = tv[q];
-                mine_row += (y.x & 0xffffu) + (y.x >> 16) + (y.y & 0xffffu) + (y.y >> 16) +
-                            (y.z & 0xffffu) + (y.z >> 16) + (y.w & 0xffffu) + (y.w >> 16);
+                if (staged) {
+                    // the entries become the survivors of the row in the warps before each one
+                    // (at most 3968), which is what the write-out needs
+                    unsigned int ws[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned int lo = ws[j] & 0xffffu, hi = ws[j] >> 16;
+                        ws[j] = mine_row | ((mine_row + lo) << 16);
+                        mine_row += lo + hi;
+                    }
+                    tv[q] = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+                } else {
+                    mine_row += (y.x & 0xffffu) + (y.x >> 16) + (y.y & 0xffffu) + (y.y >> 16) +
+                                (y.z & 0xffffu) + (y.z >> 16) + (y.w & 0xffffu) + (y.w >> 16);
+                }
             }
         }
         unsigned int run_total;
@@ -746,9 +791,30 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             if (lane == 0 && before) atomicAdd(&sh.total, before);
             __syncthreads();
             const unsigned long long base = sh.total;
-            // step 3: every warp writes the survivors of its segments that have any
+            if (staged) {
+                // step 3: one thread per survivor put aside: its place gives its index, where its
+                // value is, and its position in the output
+                const unsigned int n_st = sh.n_staged;
+                for (unsigned int j = tid; j < n_st; j += kFusedThreads) {
+                    const unsigned int tag = st_tag[j];
+                    const unsigned int r = tag >> 19, cell = (tag >> 14) & 31u, ln = (tag >> 9) & 31u, t = (tag >> 7) & 3u,
+                                       rank = tag & 127u;
+                    const long long p = (long long)base + sh.rowpre[r] + table[r * kFusedWarps + cell] + rank;
+                    if (p < cap) {
+                        const unsigned int in_row = ((cell << 5) | ln) << 2 | t;   // element within the row
+                        const int64_t at = run_lo + ((int64_t)r << 12) + in_row;
+                        const float xv = ((int)r >= first_kept)
+                                             ? reinterpret_cast<const float*>(uslot + (size_t)(r % u_slots) * kRowF4)[in_row]
+                                             : __ldcg(eps + at);
+                        idx_out[p] = (int32_t)at;
+                        val_out[p] = xv;
+                        eps[at] = 0.0f;
+                    }
+                }
+            }
+            // step 3 without the places: every warp writes the survivors of its segments that have any
             int su3 = s_run;
-            for (int cursor = 0; cursor < nrows;) {
+            for (int cursor = staged ? nrows : 0; cursor < nrows;) {
                 const int n = gather(cursor, false);
                 float4 x[kSfGroupRows];
 #pragma unroll
