@@ -89,7 +89,7 @@ k_dgck_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         ctrl->phase_t[0] = global_timer_ns();
     }
     for (int b = tid; b < kTkBins; b += kFusedThreads) sh.hist[b] = 0u;
-    if (tid == 0) { sh.need = (unsigned long long)km; sh.digit = 0u; cta_total = 0u; }
+    if (tid == 0) { sh.need = (unsigned long long)km; sh.digit = 0u; sh.n_staged = 0u; cta_total = 0u; }
     __syncthreads();
 
     // ------------------------------------------------------------------ sample: tau
@@ -340,17 +340,53 @@ k_dgck_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         // ---------------------------------------------------------- compaction
         // step 1: keys above / equal to T per marked segment; the table entry becomes
         // (above) | (equal << 8), at most 128 each
+        // The places of the entries counted here -- row, warp, lane, element, above or equal, and
+        // their ranks among the segment's keys above and equal to T -- are put aside in shared
+        // memory, two words each, as long as they fit: the write-out is then one thread per
+        // entry instead of one warp per segment.
+        unsigned int* st_ent = ACCUM ? reinterpret_cast<unsigned int*>(gring)
+                                     : reinterpret_cast<unsigned int*>(smem4 + (size_t)(kTkSmemRows - kTkStageRows) * kRowF4);
+        constexpr unsigned int kStageCap = (ACCUM ? kStages : kTkStageRows) * kRowBytes / 8;
+        const unsigned int lanes_below = (1u << lane) - 1u;
         DG_FOR_EACH_MARKED(true, {
-            unsigned int g = 0u, e = 0u;
+            unsigned int gm = 0u, em = 0u;
             if (in) {
                 const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
 #pragma unroll
-                for (int t = 0; t < 4; ++t) { g += key[t] > T; e += key[t] == T; }
+                for (int t = 0; t < 4; ++t) { gm |= (unsigned)(key[t] > T) << t; em |= (unsigned)(key[t] == T) << t; }
             }
-            const unsigned int ge = __reduce_add_sync(0xffffffffu, g | (e << 8));
+            const unsigned int ge = __reduce_add_sync(0xffffffffu, __popc(gm) | (__popc(em) << 8));
             if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)ge;
+            if (ge != 0u) {
+                const unsigned int total = (ge & 0xffu) + (ge >> 8);
+                unsigned int base = 0u;
+                if (lane == 0) base = atomicAdd(&sh.n_staged, total);
+                base = __shfl_sync(0xffffffffu, base, 0);
+                unsigned int rank_g = 0u, rank_e = 0u;
+                if (total > 1u) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        rank_g += __popc(__ballot_sync(0xffffffffu, gm & (1u << t)) & lanes_below);
+                        rank_e += __popc(__ballot_sync(0xffffffffu, em & (1u << t)) & lanes_below);
+                    }
+                }
+                if ((gm | em) && base + total <= kStageCap) {
+                    const unsigned int place = ((unsigned int)r << 19) | ((unsigned int)w << 14) | ((unsigned int)lane << 9);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const bool isg = gm & (1u << t), ise = em & (1u << t);
+                        if (isg || ise) {
+                            const unsigned int slot = base + rank_g + rank_e;
+                            st_ent[2 * slot] = place | ((unsigned int)t << 7) | (isg ? 1u : 0u);
+                            st_ent[2 * slot + 1] = rank_g | (rank_e << 8);
+                            rank_g += isg; rank_e += ise;
+                        }
+                    }
+                }
+            }
         })
         __syncthreads();
+        const bool staged = sh.n_staged <= kStageCap;
         // step 2: per row (thread t takes local row t) the two counts go to the row's words
         bool any_mine = false;
         if (tid < nrows) {
@@ -410,8 +446,39 @@ k_dgck_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
                 __syncthreads();
             }
         }
-        if (any_mine) {
-            // step 3: keys above T always, keys equal to T while fewer than need_eq came before
+        if (any_mine && staged) {
+            // step 3: one thread per entry put aside: keys above T always, keys equal to T while
+            // fewer than need_eq of them came before
+            const unsigned int n_st = sh.n_staged;
+            for (unsigned int j = tid; j < n_st; j += kFusedThreads) {
+                const unsigned int tag = st_ent[2 * j], rk = st_ent[2 * j + 1];
+                const unsigned int r = tag >> 19, cell = (tag >> 14) & 31u, ln = (tag >> 9) & 31u, t = (tag >> 7) & 3u;
+                const bool isg = tag & 1u;
+                unsigned int bg = 0u, be = 0u;   // keys above / equal to T in the warps before this one
+                for (unsigned int ww = 0; ww < cell; ++ww) {
+                    const unsigned int x = table[r * kFusedWarps + ww];
+                    bg += x & 0xffu; be += x >> 8;
+                }
+                const unsigned long long rp = sh.rowpre[r];
+                const unsigned long long ng = (rp & 0xffffffffull) + bg + (rk & 0xffu);
+                const unsigned long long ne = (rp >> 32) + be + (rk >> 8);
+                if (isg || ne < need_eq) {
+                    const unsigned long long pos = ng + (ne < need_eq ? ne : need_eq);
+                    if ((long long)pos < out_n) {
+                        const unsigned int in_row = ((cell << 5) | ln) << 2 | t;   // element within the row
+                        const int64_t at = (((int64_t)c + (int64_t)r * G) << 12) + in_row;
+                        const float x = ((int)r >= first_kept)
+                                            ? reinterpret_cast<const float*>(uslot + (size_t)(r % u_slots) * kRowF4)[in_row]
+                                            : __ldcg(reinterpret_cast<const float*>(uglob) + at);
+                        idx_out[pos] = (int32_t)at;
+                        val_out[pos] = x;
+                        if (ACCUM) eps[at] = 0.0f;
+                    }
+                }
+            }
+        } else if (any_mine) {
+            // step 3 without the places: every warp writes the selected entries of its segments
+            // that have any
             DG_FOR_EACH_MARKED(false, {
                 unsigned int gm = 0u, em = 0u;
                 if (in) {
@@ -550,8 +617,9 @@ static int enqueue_dgck(const float* src, float* eps, int64_t d, int64_t k, cons
     if (most > kTkTableMaxRows) return GK_ERR_LIMIT;
     int n_rows = (int)rows;
     const bool accum = eps != nullptr;
-    int u_slots = accum ? kTkSmemRows - DgStages<true>::value : kTkSmemRows;
-    static_assert(kTkSmemRows - DgStages<true>::value >= DgStages<true>::value && kTkSmemRows >= DgStages<false>::value,
+    // with u given there is no g ring to reuse: two rows are set aside for the places of the selected entries
+    int u_slots = accum ? kTkSmemRows - DgStages<true>::value : kTkSmemRows - kTkStageRows;
+    static_assert(kTkSmemRows - DgStages<true>::value >= DgStages<true>::value && kTkSmemRows - kTkStageRows >= DgStages<false>::value,
                   "not enough row slots for the rows in flight");
     if (u_slots > most) u_slots = (int)most;
     int64_t km = (k * m + d - 1) / d;  // the density k/d applied to the sample size

@@ -17,6 +17,9 @@ constexpr int kTkSmemBytes = kTkSmemRows * kRowBytes + kTkTableBytes;  // g ring
 template <bool ACCUM> struct TkStages { static constexpr int value = ACCUM ? 4 : 8; };
 constexpr int kTkGroupRows = 8;                                        // rows a warp gathers per batch
 constexpr int kTkBins = 2048;
+// The write-out keeps the places of a CTA's selected entries in shared memory, two words each:
+// in rows the first pass no longer needs (the g ring) or, when u is given, in two rows set aside.
+constexpr int kTkStageRows = 2;
 constexpr unsigned short kTkPending = 0xffffu;                         // table entry: segment still to be counted
 
 struct __align__(128) TopkShared {
@@ -30,6 +33,7 @@ struct __align__(128) TopkShared {
     unsigned short qrow[kFusedWarps][kTkGroupRows];
     unsigned long long need;         // entries still to take among the keys that match the digits so far
     unsigned int digit;
+    unsigned int n_staged;           // selected entries whose places were put aside for the write-out
     int ok;
 };
 static_assert((sizeof(TopkShared) + 1023) / 1024 * 1024 + kTkSmemBytes <= 232448,

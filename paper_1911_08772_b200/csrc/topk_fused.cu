@@ -82,7 +82,7 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         if (nnz_out != nullptr) *nnz_out = k;
     }
     for (int b = tid; b < kTkBins; b += kFusedThreads) sh.hist[b] = 0u;
-    if (tid == 0) { sh.need = (unsigned long long)k; sh.digit = 0u; }
+    if (tid == 0) { sh.need = (unsigned long long)k; sh.digit = 0u; sh.n_staged = 0u; }
     __syncthreads();
 
     // up to kTkGroupRows rows of this warp whose table entry is pending (want_pending) or
@@ -267,17 +267,53 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         // ---------------------------------------------------------- compaction
         // step 1: every warp counts the keys above / equal to T of its marked segments; the
         // table entry becomes (above) | (equal << 8), at most 128 each
+        // The places of the entries counted here -- row, warp, lane, element, above or equal, and
+        // their ranks among the segment's keys above and equal to T -- are put aside in shared
+        // memory, two words each, as long as they fit: the write-out is then one thread per
+        // entry instead of one warp per segment.
+        unsigned int* st_ent = ACCUM ? reinterpret_cast<unsigned int*>(gring)
+                                     : reinterpret_cast<unsigned int*>(smem4 + (size_t)(kTkSmemRows - kTkStageRows) * kRowF4);
+        constexpr unsigned int kStageCap = (ACCUM ? kStages : kTkStageRows) * kRowBytes / 8;
+        const unsigned int lanes_below = (1u << lane) - 1u;
         TK_FOR_EACH_MARKED(true, {
-            unsigned int g = 0u, e = 0u;
+            unsigned int gm = 0u, em = 0u;
             if (in) {
                 const unsigned int key[4] = {tk_key(v.x), tk_key(v.y), tk_key(v.z), tk_key(v.w)};
 #pragma unroll
-                for (int t = 0; t < 4; ++t) { g += key[t] > T; e += key[t] == T; }
+                for (int t = 0; t < 4; ++t) { gm |= (unsigned)(key[t] > T) << t; em |= (unsigned)(key[t] == T) << t; }
             }
-            const unsigned int ge = __reduce_add_sync(0xffffffffu, g | (e << 8));
+            const unsigned int ge = __reduce_add_sync(0xffffffffu, __popc(gm) | (__popc(em) << 8));
             if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)ge;
+            if (ge != 0u) {
+                const unsigned int total = (ge & 0xffu) + (ge >> 8);
+                unsigned int base = 0u;
+                if (lane == 0) base = atomicAdd(&sh.n_staged, total);
+                base = __shfl_sync(0xffffffffu, base, 0);
+                unsigned int rank_g = 0u, rank_e = 0u;
+                if (total > 1u) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        rank_g += __popc(__ballot_sync(0xffffffffu, gm & (1u << t)) & lanes_below);
+                        rank_e += __popc(__ballot_sync(0xffffffffu, em & (1u << t)) & lanes_below);
+                    }
+                }
+                if ((gm | em) && base + total <= kStageCap) {
+                    const unsigned int place = ((unsigned int)r << 19) | ((unsigned int)w << 14) | ((unsigned int)lane << 9);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const bool isg = gm & (1u << t), ise = em & (1u << t);
+                        if (isg || ise) {
+                            const unsigned int slot = base + rank_g + rank_e;
+                            st_ent[2 * slot] = place | ((unsigned int)t << 7) | (isg ? 1u : 0u);
+                            st_ent[2 * slot + 1] = rank_g | (rank_e << 8);
+                            rank_g += isg; rank_e += ise;
+                        }
+                    }
+                }
+            }
         })
         __syncthreads();
+        const bool staged = sh.n_staged <= kStageCap;
         // step 2: per row (thread t takes local row t) the two counts go to the row's words in
         // global memory; every row of the vector gets them from the CTA that owns it
         bool any_mine = false;
@@ -345,9 +381,39 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
                 __syncthreads();
             }
         }
-        if (any_mine) {
-            // step 3: every warp writes the selected entries of its segments that have any: keys
-            // above T always, keys equal to T while fewer than need_eq of them came before
+        if (any_mine && staged) {
+            // step 3: one thread per entry put aside: keys above T always, keys equal to T while
+            // fewer than need_eq of them came before
+            const unsigned int n_st = sh.n_staged;
+            for (unsigned int j = tid; j < n_st; j += kFusedThreads) {
+                const unsigned int tag = st_ent[2 * j], rk = st_ent[2 * j + 1];
+                const unsigned int r = tag >> 19, cell = (tag >> 14) & 31u, ln = (tag >> 9) & 31u, t = (tag >> 7) & 3u;
+                const bool isg = tag & 1u;
+                unsigned int bg = 0u, be = 0u;   // keys above / equal to T in the warps before this one
+                for (unsigned int ww = 0; ww < cell; ++ww) {
+                    const unsigned int x = table[r * kFusedWarps + ww];
+                    bg += x & 0xffu; be += x >> 8;
+                }
+                const unsigned long long rp = sh.rowpre[r];
+                const unsigned long long ng = (rp & 0xffffffffull) + bg + (rk & 0xffu);
+                const unsigned long long ne = (rp >> 32) + be + (rk >> 8);
+                if (isg || ne < need_eq) {
+                    const unsigned long long pos = ng + (ne < need_eq ? ne : need_eq);
+                    if ((long long)pos < k) {
+                        const unsigned int in_row = ((cell << 5) | ln) << 2 | t;   // element within the row
+                        const int64_t at = (((int64_t)c + (int64_t)r * G) << 12) + in_row;
+                        const float x = ((int)r >= first_kept)
+                                            ? reinterpret_cast<const float*>(uslot + (size_t)(r % u_slots) * kRowF4)[in_row]
+                                            : __ldcg(reinterpret_cast<const float*>(uglob) + at);
+                        idx_out[pos] = (int32_t)at;
+                        val_out[pos] = x;
+                        if (ACCUM) eps[at] = 0.0f;
+                    }
+                }
+            }
+        } else if (any_mine) {
+            // step 3 without the places: every warp writes the selected entries of its segments
+            // that have any
             TK_FOR_EACH_MARKED(false, {
                 unsigned int gm = 0u, em = 0u;
                 if (in) {
@@ -493,8 +559,9 @@ int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, i
     int n_rows = (int)rows;
     const bool accum = eps != nullptr;
     // a slot is reused kStages - 1 rows later at the earliest: u_slots >= kStages in both forms
-    int u_slots = accum ? kTkSmemRows - TkStages<true>::value : kTkSmemRows;
-    static_assert(kTkSmemRows - TkStages<true>::value >= TkStages<true>::value && kTkSmemRows >= TkStages<false>::value,
+    // with u given there is no g ring to reuse: two rows are set aside for the places of the selected entries
+    int u_slots = accum ? kTkSmemRows - TkStages<true>::value : kTkSmemRows - kTkStageRows;
+    static_assert(kTkSmemRows - TkStages<true>::value >= TkStages<true>::value && kTkSmemRows - kTkStageRows >= TkStages<false>::value,
                   "not enough row slots for the rows in flight");
     if (u_slots > most) u_slots = (int)most;
     Ctrl* ctrl = ws->ctrl;
