@@ -264,8 +264,8 @@ int gk_histogram(const float* u, int64_t d, float lo, float inv_w, int32_t nbins
  * Limits: 1 <= k < d <= 2^31 - 1 (d beyond that returns GK_ERR_SIZE; k = d
  * returns GK_ERR_K: selecting everything is left to gk_sparsify); the device
  * must support cooperative launch, the launch must fit the array's 512
- * per-CTA slots, and the vector must not exceed 448 rows of 4096 elements per
- * SM (271 M elements on 148 SMs), else GK_ERR_LIMIT.
+ * per-CTA slots, and the vector must not exceed 2^29 elements (the array has one
+ * word per row of 4096 elements) nor 1024 rows per SM, else GK_ERR_LIMIT.
  *
  * The first call on a device looks up the array's device address
  * (cudaGetSymbolAddress) and keeps it; make that first call before any stream

@@ -43,9 +43,9 @@
 
 namespace gk {
 
-constexpr int kTableMaxRows = 448;                     // most rows a CTA may own (entries of its maximum table)
+constexpr int kTableMaxRows = 1024;                    // most rows a CTA may own (entries of its maximum table)
 constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, warp)
-constexpr int kFusedSmemBudget = 226304;               // dynamic shared memory the kernel may ask for
+constexpr int kFusedSmemBudget = 221184;               // dynamic shared memory the kernel may ask for
 constexpr int kStages = 4;                             // phase A: rows of g and eps in flight, plus one
 constexpr int kRing = 8;                               // ring slots; phase B has kRing - 1 rows in flight
 constexpr int kGroupRows = 8;                          // rows a warp gathers per batch in phase C
@@ -138,10 +138,17 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
         // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
         int64_t fi = first4;  // the row the next fetch brings in
+        // Where the eps of local row r lands.  Normally the slot that will hold u.  A CTA with so
+        // many rows that its table leaves fewer slots than rows in flight takes eps through the
+        // half of the ring that g does not use, and only its last rows are kept on chip.
+        const bool eps_ring = u_slots < kStages;
+        auto eps_slot = [&](int r) -> float4* {
+            return eps_ring ? gring + (size_t)(kStages + r % kStages) * kRowF4 : uslot + (size_t)(r % u_slots) * kRowF4;
+        };
         auto fetch = [&](int r) {
             if (r < nrows && fi < n4) {
                 cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
-                cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + fi);
+                cp_async16(eps_slot(r) + tid, e4 + fi);
             }
             cp_async_commit();
             fi += stride4;
@@ -155,10 +162,11 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             const bool one = i < n4;
             float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one) {
-                float4* us = uslot + (size_t)(r % u_slots) * kRowF4 + tid;
-                const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *us;
+                float4* es = eps_slot(r) + tid;
+                const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *es;
                 u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
-                *us = u0;
+                if (!eps_ring) *es = u0;
+                else if (r >= first_kept) uslot[(size_t)(r % u_slots) * kRowF4 + tid] = u0;
                 const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
                              x3 = (double)u0.w - pv;
                 s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
@@ -687,9 +695,9 @@ static FusedGeometry fused_geometry(int64_t d, int grid) {
     const int64_t left = (int64_t)kFusedSmemBudget - (int64_t)kRing * kRowBytes - (int64_t)q.table_rows * kTableRowBytes;
     q.u_slots = (int)(left / kRowBytes);
     if (q.u_slots > most) q.u_slots = (int)most;
-    // a slot is written again kStages - 1 rows later: with fewer slots than rows in flight the
-    // copy for a later row would land on the row being read
-    if (q.u_slots < kStages && q.u_slots < most) q.fits = false;
+    // (with fewer slots than rows in flight the kernel takes eps through the ring instead; the
+    // last row of the vector, which may be short, must stay on chip: one slot at least)
+    if (q.u_slots < 1) q.fits = false;
     q.smem = (size_t)(kRing + q.u_slots) * kRowBytes + (size_t)q.table_rows * kTableRowBytes;
     return q;
 }

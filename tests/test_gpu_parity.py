@@ -435,3 +435,24 @@ def test_workload_sweep_largest(dist):
     ties_all = np.nonzero(np.abs(g) == kth)[0]
     ties_sel = hi[np.abs(hv) == kth]
     assert np.array_equal(ties_sel, ties_all[:ties_sel.size].astype(np.int32))
+
+
+def test_gk_half_a_billion_elements_on_the_fused_kernel():
+    """d = 2^29 + 3 (the upper end of the paper's operator timing sweep, Section 4.1): 886 rows
+    per CTA, eps taken through the ring, one row kept on chip, a ragged tail; against the
+    oracle in full."""
+    d = (1 << 29) + 3
+    k = wl.ceil_k(d, 1, 1000)
+    g = wl.normal(d, 1.0, step=11)
+    z = np.zeros(d, dtype=np.float32)
+    cap = 2 * k
+    gk.gk_set_capacity(cap)
+    try:
+        step = DeviceStep(d, cap=cap)
+        before = gk.gk_launch_count()
+        check_gk_step(step, g, z, k)
+        assert gk.gk_launch_count() - before == 1      # one cooperative kernel, not the three-kernel form
+    finally:
+        gk.gk_set_capacity(0)
+    del step
+    torch.cuda.empty_cache()
