@@ -115,34 +115,48 @@ __device__ inline Alg1Path alg1_replay(const unsigned long long* counts, int64_t
     Alg1Path p;
     p.chosen = 0;
     p.rounds = 0;
-    for (int r = 0; r < kMaxRounds; ++r) p.est[r] = 0;
     int h = 0, b = 0;
+    bool going = true;
+    // four rounds at most, written out so that nothing is indexed by a run-time value (arrays
+    // indexed that way live in local memory, and one thread walks this chain for the whole grid)
+#pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
-        const int ci = cand_index(h, b);
-        // the counts may live in global or in shared memory: a generic volatile load serves both
-        const long long est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&counts[ci]);
+        long long est = 0;
+        if (going) {
+            const int ci = cand_index(h, b);
+            // the counts may live in global or in shared memory: a generic volatile load serves both
+            est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&counts[ci]);
+            p.rounds = r + 1;
+            p.chosen = ci;
+            if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
+            else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
+            else going = false;
+        }
         p.est[r] = est;
-        p.rounds = r + 1;
-        p.chosen = ci;
-        if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
-        else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
-        else break;
     }
     return p;
+}
+
+// The count of the last round that ran (the size of the returned mask).
+__device__ inline long long alg1_last_est(const Alg1Path& p) {
+    long long last = p.est[0];
+#pragma unroll
+    for (int r = 1; r < kMaxRounds; ++r) if (r < p.rounds) last = p.est[r];
+    return last;
 }
 
 // The same with the record filled in.  One thread.
 // Returns the index of the candidate whose mask is returned (-1: everything).
 __device__ inline int alg1_resolve(const Alg1State& a, int64_t k) {
-    gk_stats st = *a.stats;
-    if (st.rounds == 0 && st.thr_final == -INFINITY) return -1;  // everything selected
+    gk_stats* st = a.stats;
+    if (st->rounds == 0 && st->thr_final == -INFINITY) return -1;  // everything selected
     const Alg1Path p = alg1_replay(a.counts, k);
-    for (int r = 0; r < p.rounds; ++r) st.counts[r] = p.est[r];
-    st.rounds = p.rounds;
-    st.thr_final = a.cand64[p.chosen];  // the mask of the last round evaluated
-    st.nnz = p.est[p.rounds - 1];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) st->counts[r] = p.est[r];   // rounds not run keep 0
+    st->rounds = p.rounds;
+    st->thr_final = a.cand64[p.chosen];  // the mask of the last round evaluated
+    st->nnz = alg1_last_est(p);
     *a.thr_sel = a.cand32[p.chosen];
-    *a.stats = st;
     return p.chosen;
 }
 #endif

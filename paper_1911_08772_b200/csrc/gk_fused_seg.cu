@@ -574,7 +574,7 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
                     float t = INFINITY;
                     for (int j = 0; j < kNumCand; ++j) if (sh.ord[q][j] == p.chosen) t = sh.cs[q][j];
                     sh.thr[q] = t;
-                    nz = (unsigned long long)p.est[p.rounds - 1];
+                    nz = (unsigned long long)alg1_last_est(p);
                 } else {
                     nz = (unsigned long long)n;  // everything selected
                 }
@@ -889,10 +889,11 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             for (int j = 0; j < kNumCand; ++j) cnt[j] = __ldcg(&v.counts[(size_t)q * kNumCand + j]);
             gk_stats rec = v.stats[q];
             const Alg1Path p = alg1_replay(cnt, kk);
-            for (int r = 0; r < p.rounds; ++r) rec.counts[r] = p.est[r];
+#pragma unroll
+            for (int r = 0; r < kMaxRounds; ++r) rec.counts[r] = p.est[r];   // rounds not run: 0
             rec.rounds = p.rounds;
             rec.thr_final = v.cand64[(size_t)q * kNumCand + p.chosen];
-            rec.nnz = p.est[p.rounds - 1];
+            rec.nnz = alg1_last_est(p);
             v.stats[q] = rec;
             v.thr_sel[q] = sh.thr[q];
         }
