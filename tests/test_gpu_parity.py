@@ -456,3 +456,24 @@ def test_gk_half_a_billion_elements_on_the_fused_kernel():
         gk.gk_set_capacity(0)
     del step
     torch.cuda.empty_cache()
+
+
+def test_everything_selected_on_a_vector_of_many_rows(gk_path):
+    """A mean far below zero makes every threshold of Algorithm 1 negative, so every element is
+    selected: more survivors per CTA than the on-chip list of places holds, which takes the
+    write-out of one warp per segment; whole vector and layer-wise."""
+    d = 6_000_003
+    rng = wl.misc_rng(77)
+    g = (rng.standard_normal(d) * 1e-3 - 5.0).astype(np.float32)
+    z = np.zeros(d, dtype=np.float32)
+    step = DeviceStep(d)
+    eps_new, st = check_gk_step(step, g, z, 6000)
+    assert st.nnz == d and st.thr_final < 0 and not eps_new.any()
+    if gk_path == 0:
+        offsets = np.array([0, 1_000_001, 1_000_001, 3_500_000, d], dtype=np.int64)
+        seg_k = np.array([1000, 5, 2500, 2500], dtype=np.int64)
+        dev_off = torch.from_numpy(offsets).cuda()
+        dev_k = torch.from_numpy(seg_k).cuda()
+        nn = torch.zeros(4, dtype=torch.int64, device="cuda")
+        eps_new, _ = check_segmented_step(step, g, z, offsets, seg_k, dev_off, dev_k, nn)
+        assert not eps_new.any()
