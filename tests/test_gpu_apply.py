@@ -112,7 +112,7 @@ def test_apply_after_real_sparsifier_steps(P):
 
 
 def test_exchange_and_apply_through_nccl_with_one_rank():
-    """The wrapper end to end on the GPU: a one-rank NCCL group (this box has one GPU), the
+    """The wrapper end to end on the GPU: a one-rank NCCL group (one GPU is enough), the
     all-gather of the message, the update kernel; against the oracle."""
     import os
     import socket
