@@ -460,6 +460,38 @@ def run_ours(args):
                    "(no all-gather in this number)")
     del x_model, eps4
 
+    # ---- the layer-wise (segmented) call on the same data, where the workload has segments:
+    # episodes of 4 steps from eps = 0
+    seg = None
+    if w.partition is not None:
+        part = w.partition
+        seg = {}
+        d_off = torch.from_numpy(part.offsets).to(dev)
+        seg_nnz = torch.zeros(part.S, dtype=torch.int64, device=dev)
+        eps5 = torch.zeros_like(epss[0])
+        gk.gk_reserve(d, part.S)
+        for rho_s in ("1e-3", "1e-2"):
+            d_k = torch.from_numpy(part.seg_k(*wl.RHO[rho_s])).to(dev)
+
+            def seg_step(t, d_k=d_k):
+                gk.gk_sparsify_segmented(gs[t % n_rot], eps5, d_off, d_k, idx, val, seg_nnz, nnz)
+
+            eps5.zero_()
+            for t in range(4):
+                seg_step(t)
+            ms_seg, n_seg = 0.0, 0
+            for e in range(10):
+                eps5.zero_()
+                ms_seg += time_region(torch, seg_step, 4)
+                n_seg += 4
+            ms_seg /= n_seg
+            nz = float(nnz.item())
+            seg[f"rho={rho_s}"] = {"ms": ms_seg, "nnz_last": nz, "gbs": algorithmic_bytes(d, nz) / ms_seg / 1e6,
+                                   "frac_of_measured_hbm": algorithmic_bytes(d, nz) / ms_seg / 1e6 / peak}
+        seg["segments"] = part.S
+        seg["call"] = "gk_sparsify_segmented, one cooperative kernel, k_s = ceil(rho * d_s)"
+        del eps5
+
     # ---- the error ratio of Eq. 5 for one Gaussian_k step and one Top_k step from eps = 0
     diag = {"bound_eq4_1_minus_k_over_d": 1.0 - k / d, "bound_theorem1_squared": (1.0 - k / d) ** 2}
     eps3 = torch.zeros_like(epss[0])
@@ -536,7 +568,7 @@ def run_ours(args):
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
                  "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
-        "dgck": dgck, "update_from_messages": upd, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
+        "segmented": seg, "dgck": dgck, "update_from_messages": upd, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
         "clocks": sampler.summary(),
     }
     print(json.dumps(line))
