@@ -105,34 +105,37 @@ int64_t oracle_count_above(const float* u, int64_t d, double thres) {
 }
 
 // ---------------------------------------------------------------------------
-// Alg. 1 up to the end of its loop: statistics, initial threshold, and the
-// count-and-adjust rounds.
-// Fills st (everything except nnz is final on return; nnz = last count).
+// Algorithm 1 up to the end of its loop.  The first threshold is the normal quantile at
+// probability 1 - k/d for the vector's own mean and deviation.  Then, at most four times: count
+// the magnitudes above the threshold; fewer than two thirds of k halves the threshold, more
+// than four thirds of k multiplies it by 1.5 (both tested exactly in integers), anything
+// between ends the loop.  The mask that is returned is the one of the last count taken, so
+// thr_final and nnz record that round and an adjustment made after it is dropped.
 // ---------------------------------------------------------------------------
 void oracle_gaussiank_threshold(const float* u, int64_t d, int64_t k, int max_rounds,
                                 int unbiased, oracle_stats* st) {
     std::memset(st, 0, sizeof(*st));
-    if (k >= d) {  // p = 1 - k/d <= 0: the quantile is -inf, every element passes
+    if (k >= d) {  // the probability is <= 0: the quantile is -inf, every element passes
         st->mu = st->sigma = std::numeric_limits<double>::quiet_NaN();
         st->z = st->thres0 = st->thr_final = -std::numeric_limits<double>::infinity();
         st->rounds = 0;
         st->nnz = d;
         return;
     }
-    oracle_mean_std(u, d, unbiased, &st->mu, &st->sigma);       // mu, sigma
-    const double p = 1.0 - (double)k / (double)d;               // p = 1 - k/d
+    oracle_mean_std(u, d, unbiased, &st->mu, &st->sigma);
+    const double p = 1.0 - (double)k / (double)d;
     st->z = oracle_norm_ppf(p);
-    double thres = st->mu + st->sigma * st->z;                  // ppf(p; mu, sigma)
+    double thres = st->mu + st->sigma * st->z;
     st->thres0 = thres;
     if (max_rounds > 4) max_rounds = 4;
-    for (int i = 0; i < max_rounds; ++i) {                      // i = 0 .. 3
-        const int64_t est = oracle_count_above(u, d, thres);    // estimated_k
+    for (int i = 0; i < max_rounds; ++i) {
+        const int64_t est = oracle_count_above(u, d, thres);
         st->counts[i] = est;
         st->rounds = i + 1;
-        st->thr_final = thres;  // the mask of this round is the last one evaluated
+        st->thr_final = thres;
         st->nnz = est;
-        if (3 * est < 2 * k) thres = 0.5 * thres;               // est < 2k/3
-        else if (3 * est > 4 * k) thres = 1.5 * thres;          // est > 4k/3
+        if (3 * est < 2 * k) thres = 0.5 * thres;
+        else if (3 * est > 4 * k) thres = 1.5 * thres;
         else break;
     }
 }

@@ -24,6 +24,8 @@
 //
 // Rows of 1024 float4 are dealt to one CTA per SM in turn, as in the other
 // persistent kernels.  All waits are bounded (grid_barrier).
+#include <mutex>
+
 #include "gk_common.cuh"
 #include "gk_coop.cuh"
 #include "gk_radix.cuh"
@@ -586,6 +588,9 @@ static bool dgck_kernel_ready() {
 
 static DgPlan* dgck_plan(int dev, int sm_count) {
     if (dev < 0 || dev >= 64) return nullptr;
+    // built once per device, under a lock: a second thread's first call waits for the finished plan
+    static std::mutex plan_mu;
+    std::lock_guard<std::mutex> plan_lock(plan_mu);
     DgPlan& p = g_dg_plan[dev];
     if (p.ready) return &p;
     p.ready = true;

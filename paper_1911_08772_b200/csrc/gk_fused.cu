@@ -650,6 +650,9 @@ static FusedPlan g_plan[64];
 
 static FusedPlan* fused_plan(int dev, int sm_count) {
     if (dev < 0 || dev >= 64) return nullptr;
+    // built once per device, under a lock: a second thread's first call waits for the finished plan
+    static std::mutex plan_mu;
+    std::lock_guard<std::mutex> plan_lock(plan_mu);
     FusedPlan& p = g_plan[dev];
     if (p.ready) return &p;
     p.ready = true;

@@ -26,6 +26,8 @@
 // without cooperative launch take the three-kernel form in gk_segmented.cu.
 #include <math.h>
 
+#include <mutex>
+
 #include "gk_alg1.cuh"
 #include "gk_common.cuh"
 #include "gk_coop.cuh"
@@ -925,6 +927,9 @@ static SegFusedPlan g_sf_plan[64];
 
 static SegFusedPlan* seg_fused_plan(int dev, int sm_count) {
     if (dev < 0 || dev >= 64) return nullptr;
+    // built once per device, under a lock: a second thread's first call waits for the finished plan
+    static std::mutex plan_mu;
+    std::lock_guard<std::mutex> plan_lock(plan_mu);
     SegFusedPlan& p = g_sf_plan[dev];
     if (p.ready) return &p;
     p.ready = true;

@@ -86,7 +86,10 @@ int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out
         void* p = nullptr;
         cudaError_t e = cudaMalloc(&p, L.total);
         if (e != cudaSuccess) { cudaGetLastError(); return GK_ERR_NOMEM; }
-        e = cudaMemset(p, 0, L.total);
+        // cleared on the caller's stream, so that the clear is ordered before the kernels of this and
+        // every later call there (a memset on the default stream would not be ordered with a
+        // non-blocking stream)
+        e = cudaMemsetAsync(p, 0, L.total, stream);
         if (e != cudaSuccess) { cudaFree(p); return cuda_fail(e); }
         char* b = static_cast<char*>(p);
         ws.base = p;
@@ -255,11 +258,10 @@ extern "C" int gk_sparsify_host(const float* g, float* eps, int64_t d, int64_t k
     int dev = 0;
     GK_CUDA_TRY(cudaGetDevice(&dev));
     const int64_t cap = output_capacity(d);
-    HostStage* hs;
-    {
-        std::lock_guard<std::mutex> lock(g_mu);
-        hs = &g_stage[dev];
-    }
+    // the staging buffers of a device serve one call at a time
+    static std::mutex stage_mu;
+    std::lock_guard<std::mutex> stage_lock(stage_mu);
+    HostStage* hs = &g_stage[dev];
     if (!hs->stream) GK_CUDA_TRY(cudaStreamCreateWithFlags(&hs->stream, cudaStreamNonBlocking));
     if (d > hs->d_cap || cap > hs->out_cap) {
         GK_CUDA_TRY(cudaStreamSynchronize(hs->stream));

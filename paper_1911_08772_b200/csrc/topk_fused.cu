@@ -28,6 +28,8 @@
 // GK_DEV_TIMEOUT and leaves.  Vectors whose runs exceed the table (more than
 // kTkTableMaxRows rows per CTA) and devices without cooperative launch take
 // the multi-kernel path in topk_exact.cu.
+#include <mutex>
+
 #include "gk_common.cuh"
 #include "gk_coop.cuh"
 #include "gk_count.cuh"
@@ -525,6 +527,9 @@ static bool topk_kernel_ready(int sm_count) {
 
 static TopkPlan* topk_plan(int dev, int sm_count) {
     if (dev < 0 || dev >= 64) return nullptr;
+    // built once per device, under a lock: a second thread's first call waits for the finished plan
+    static std::mutex plan_mu;
+    std::lock_guard<std::mutex> plan_lock(plan_mu);
     TopkPlan& p = g_tk_plan[dev];
     if (p.ready) return &p;
     p.ready = true;

@@ -70,18 +70,17 @@ class DeviceStep:
         return idx[:n].copy(), val[:n].copy(), n
 
 
-def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, check_counts=True):
-    """Run one gk_sparsify step on the device and compare with the oracle.
-    Returns (eps_new (numpy, from the device), stats)."""
-    d = g.shape[0]
-    step.g.copy_(torch.from_numpy(g))
-    step.eps.copy_(torch.from_numpy(eps_in))
-    step.arm()
-    gk.gk_sparsify(step.g, step.eps, k, step.idx[:step.cap], step.val[:step.cap], step.nnz[:1])
-    idx, val, n = step.outputs()
-    st = gk.gk_last_stats()
-    eps_new = step.eps.cpu().numpy()
+def compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, cap, check_counts=True):
+    """One finished sparsifier step (pairs idx/val[:n], record st, residual eps_new, output
+    capacity cap) against the oracle, by the acceptance rule in this module's header.
 
+    Two of the tolerances have an absolute alternative, for quantities that can sit at zero,
+    where a relative bound says nothing: mu against 1e-9 sigma (the mean of zero-mean data is
+    rounding noise around 0), thres0 and the final threshold against 1e-6 sigma (mu + sigma z
+    crosses zero for k near d / 2).  z is compared absolutely, 1e-12 on a quantity of order 1:
+    at p = 1/2 the oracle's bisection ends one denormal below zero where the library's Newton
+    iteration returns 0 exactly."""
+    d = g.shape[0]
     u = orc.accumulate(g, eps_in)
     ost = orc.gaussiank_threshold(u, k)
     assert st.status in (0, gk.GK_DEV_TRUNCATED)
@@ -97,14 +96,28 @@ def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, c
     else:
         assert st.rounds == 0 and st.thr_final == -math.inf
     # selection with the library's own threshold
-    oi, ov, on = orc.select(u, st.thr_final, cap=step.cap)
+    oi, ov, on = orc.select(u, st.thr_final, cap=cap)
     assert st.nnz == on
-    assert n == min(on, step.cap) == st.emitted
-    assert (st.status & gk.GK_DEV_TRUNCATED) == (gk.GK_DEV_TRUNCATED if on > step.cap else 0)
+    assert n == min(on, cap) == st.emitted
+    assert (st.status & gk.GK_DEV_TRUNCATED) == (gk.GK_DEV_TRUNCATED if on > cap else 0)
     assert np.array_equal(idx, oi)
     assert np.array_equal(bits(val), bits(ov))
     oeps = orc.residual(u, oi, ov)
     assert np.array_equal(bits(eps_new), bits(oeps))
+
+
+def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, check_counts=True,
+                  call=None):
+    """Run one gk_sparsify step (or `call`, an entry point with the same arguments) on the
+    device and compare with the oracle.  Returns (eps_new (numpy, from the device), stats)."""
+    step.g.copy_(torch.from_numpy(g))
+    step.eps.copy_(torch.from_numpy(eps_in))
+    step.arm()
+    (call or gk.gk_sparsify)(step.g, step.eps, k, step.idx[:step.cap], step.val[:step.cap], step.nnz[:1])
+    idx, val, n = step.outputs()
+    st = gk.gk_last_stats()
+    eps_new = step.eps.cpu().numpy()
+    compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, step.cap, check_counts)
     return eps_new, st
 
 

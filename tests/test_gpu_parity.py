@@ -64,7 +64,10 @@ def test_gk_sparsify_special_values(gk_path):
     z = np.zeros(d, dtype=np.float32)
     _, st = check_gk_step(step, z, z, 10)
     assert st.nnz == 0 and st.sigma == 0.0
-    # constant vector: sigma = 0
+    # constant vector: sigma = 0 and thres0 = mu, so every element sits exactly on the first
+    # threshold.  One rounding of difference in mu (the two sides sum in different orders) moves
+    # all d elements across it, so the per-round counts are not compared here; the threshold
+    # (1e-6) and the selection at the library's own threshold still are.
     c = np.full(d, 0.375, dtype=np.float32)
     check_gk_step(step, c, z, 10, check_counts=False)
     # large mean relative to the spread
