@@ -8,9 +8,14 @@ One "step" is one whole pass of the hot path -- gk_sparsify(g, eps, d, k, ...) -
 synthetic gradient vector with the residual eps carried from step to step.  The default
 workload is the ResNet-50-sized vector (d = 25,557,032, rho = 1e-3, whole-vector
 selection).  The metric is throughput in GB/s of ALGORITHMIC bytes:
-    bytes/step = 20 * d + 12 * nnz
-(read g and eps, write u over eps, one read of u for the candidate counts, one read of u
-for the compaction, 8 bytes per emitted pair and 4 per cleared residual slot).
+    bytes/step = (16 + 4 r) * d + 12 * nnz,   r = count passes over u that the step ran
+(read g and eps, write u over eps, one read of u per count pass, one read of u for the
+compaction, 8 bytes per emitted pair and 4 per cleared residual slot).  r = 1 when all ten
+candidate thresholds are counted in one pass after the statistics; r = 0 when the counts were
+taken while the vector streamed in (the kernel reports which, see gk_last_path_info).
+
+With a small --steps K the K-step region is repeated until about 0.3 s have been timed and
+the median region is reported, so that a short run and a long one measure the same thing.
 
 Printed: one JSON line.  With --impl reference the CPU oracle
 is timed instead, on the host cores, on the same workload.  With N > 1 (torchrun) every rank
@@ -39,10 +44,10 @@ UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
 N_ROTATE = 20   # distinct gradients: the workload's 20 error-compensation iterations, then again
 EPISODE = 20    # steps that share one residual buffer (eps starts at zero)
-# DRAM bytes of one k_gk_fused launch at d = 25,557,032 (248.2 MB read + 64.3 MB written), from the
-# ncu capture summarised under profiles/; valid only for the kernel as it stood at that capture
-FUSED_DRAM_BYTES_PER_LAUNCH = 312566016
-FUSED_DRAM_CAPTURE_D = 25557032
+FUSED_PROFILE = os.path.join(ROOT, "profiles", "k_gk_fused_resnet50_ncu_full.txt")
+# files whose contents decide what k_gk_fused does: the ncu figures hold only for these
+FUSED_SOURCES = ["gk_fused.cu", "gk_coop.cuh", "gk_count.cuh", "gk_alg1.cuh", "gk_common.cuh"]
+MIN_TIMED_MS = 300.0   # the timed region is repeated until this much has been timed
 MAX_EPS = 48    # residual buffers kept (pre-zeroed); beyond that they are reused as they stand
 
 
@@ -54,8 +59,35 @@ def measured_peaks():
     return 6650.0, "fallback (earlier measurement on this pool)"
 
 
-def algorithmic_bytes(d: int, nnz: float) -> float:
-    return 20.0 * d + 12.0 * nnz
+def algorithmic_bytes(d: int, nnz: float, r: float = 1.0) -> float:
+    """(16 + 4 r) d + 12 nnz: r = count passes over u (1: one pass for all ten candidates)."""
+    return (16.0 + 4.0 * r) * d + 12.0 * nnz
+
+
+def fused_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in FUSED_SOURCES:
+        with open(os.path.join(ROOT, "paper_1911_08772_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(d: int):
+    """DRAM bytes per launch of k_gk_fused from the committed ncu summary, or None when that
+    capture was of another size or of other kernel sources."""
+    try:
+        rec = {}
+        with open(FUSED_PROFILE) as f:
+            for line in f:
+                if ":" in line:
+                    key, _, v = line.partition(":")
+                    rec[key.strip()] = v.strip()
+        if int(rec["capture_d"]) != d or rec["kernel_source_sha256_16"] != fused_source_hash():
+            return None
+        return int(rec["dram_bytes_per_launch"])
+    except Exception:
+        return None
 
 
 def pick_workload(name: str):
@@ -149,9 +181,13 @@ def cpu_oracle_rate(w, rho, steps: int, warmup: int = 0):
         dt = time.perf_counter() - t0
         if t >= warmup:
             total_t += dt
-            total_b += algorithmic_bytes(w.d, idx.size)
+            total_b += algorithmic_bytes(w.d, idx.size, st.rounds)   # the oracle reads u once per round
         nnz_last = idx.size
     return total_b / total_t / 1e9, total_t / steps, nnz_last
+
+
+def workload_string(w, rho) -> str:
+    return f"{w.name} d={w.d} rho={rho} k={w.k(rho)} whole-vector selection, eps carried over"
 
 
 def run_reference(args):
@@ -161,13 +197,14 @@ def run_reference(args):
     w, rho = pick_workload(args.workload)
     # each oracle step at d = 25.6M takes ~0.5 s on one core: bound the run to a few minutes
     steps = max(1, min(args.steps, 60))
-    warm = max(0, min(args.warmup, 3))
+    warm = max(0, min(args.warmup, 20))
     gbs, s_per_step, nnz = cpu_oracle_rate(w, rho, steps, warm)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": steps, "warmup": warm, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": warm, "ms_per_step": s_per_step * 1e3, "steps_per_s": 1.0 / s_per_step,
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name} d={w.d} rho={rho} k={w.k(rho)} whole-vector selection",
+        "config": {"workload": workload_string(w, rho),
                    "note": "CPU oracle (oracle/gk_oracle.cpp), one thread"},
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{steps} full steps of the workload (requested {args.steps})"},
@@ -274,6 +311,9 @@ def run_ours(args):
             else:
                 def step(t):  # noqa: F811
                     gk.dgck_select(gs[t % n_rot], k, smp, idx, val, nnz)
+        elif args.call == "gk_select":
+            def step(t):  # noqa: F811
+                gk.gk_select(gs[t % n_rot], k, idx, val, nnz)
         else:
             def step(t):  # noqa: F811
                 gk.topk_exact(gs[t % n_rot], k, idx, val)
@@ -287,15 +327,26 @@ def run_ours(args):
     for t in range(W):
         step(t)
     barrier()
+    # the K-step region, repeated until MIN_TIMED_MS have been timed (the same number of
+    # repeats on every rank); the median region is the one reported
     launches0 = gk.gk_launch_count()
     sampler = ClockSampler(local)
+    regions = []
     with sampler:
-        ms = time_region(torch, lambda t: step(W + t), K)
+        first = max_over_ranks(time_region(torch, lambda t: step(W + t), K), world, dev)
+        regions.append(first)
+        repeats = 1 if args.loop_only else max(1, min(2000, int(MIN_TIMED_MS / max(first, 1e-3)) + 1))
+        for rep in range(1, repeats):
+            barrier()
+            regions.append(max_over_ranks(time_region(torch, lambda t: step(W + rep * K + t), K), world, dev))
     barrier()
-    launches = gk.gk_launch_count() - launches0
-    ms = max_over_ranks(ms, world, dev)
+    launches = (gk.gk_launch_count() - launches0) // len(regions)
+    ms = statistics.median(regions)
     nnz_mean = float(nnz.item())  # of the last step; 12 * nnz is ~0.03 % of the bytes
-    bytes_step = algorithmic_bytes(d, nnz_mean)
+    # how the last step took its counts: r = 0 when every CTA counted while streaming
+    info = gk.gk_last_path_info() if args.call == "gk" and args.path == 0 else (0, 0, 0, 0, 0)
+    r_passes = (0.0 if info[4] > 0 and info[1] == info[4] else 1.0) + (1.0 if info[2] else 0.0)
+    bytes_step = algorithmic_bytes(d, nnz_mean, r_passes)
     value = whole_job_gbs(world, bytes_step, K, ms)
     peak, peak_src = measured_peaks()
 
@@ -305,7 +356,8 @@ def run_ours(args):
         return
     if args.loop_only:
         print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-                          "warmup": W, "ms_per_step": ms / K, "path": args.path, "loop_only": True}))
+                          "warmup": W, "ms_per_step": ms / K, "path": args.path, "loop_only": True,
+                          "count_passes": r_passes, "path_info": info}))
         return
 
     # ---- per-kernel durations (CUDA events recorded by the library around its kernels)
@@ -322,17 +374,36 @@ def run_ours(args):
 
     fused = stage_means(7)
     fused_ms = float(fused[0])
+    traffic = recorded_traffic(d)
     roof = {
         "bound": "hbm", "kernel": "k_gk_fused", "achieved": bytes_step / (fused_ms * 1e-3) / 1e9,
         "peak": peak, "unit": "GB/s", "peak_source": peak_src,
         "frac": bytes_step / (fused_ms * 1e-3) / 1e9 / peak,
-        "traffic": FUSED_DRAM_BYTES_PER_LAUNCH if d == FUSED_DRAM_CAPTURE_D else None,
+        "frac_of_nominal_8TBs": bytes_step / (fused_ms * 1e-3) / 1e9 / 8000.0,
+        "traffic": traffic,
         "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of k_gk_fused at this d "
-                          "(profiles/k_gk_fused_resnet50_ncu_full.txt)",
+                          "(profiles/k_gk_fused_resnet50_ncu_full.txt); null when the kernel's sources have "
+                          "changed since that capture",
         "kernel_ms": fused_ms,
+        "kernel_ms_source": "mean over %d launches of CUDA events the library records around the kernel on its "
+                            "stream, one launch at a time (a second loop right after the headline loop, whose "
+                            "back-to-back launches overlap their ends and starts: ms_per_step is smaller)" % Ks,
         "phase_ms": {"accumulate_stats+barrier": fused[1], "count_loop": fused[2], "barrier2": fused[3],
                      "replay_rounds": fused[4], "compact": fused[5], "last_cta_exit": fused[6]},
         "bytes_per_launch": bytes_step,
+        "bytes_model": f"(16 + 4 r) d + 12 nnz with r = {r_passes:g} count passes over u",
+        # what DRAM really moved, against both peaks: the counts and most of the compaction are
+        # served from shared memory and L2, so this is below the algorithmic rate
+        "dram": None if traffic is None else {
+            "bytes_per_launch": traffic, "gbs": traffic / (fused_ms * 1e-3) / 1e9,
+            "frac_of_measured_copy": traffic / (fused_ms * 1e-3) / 1e9 / peak,
+            "frac_of_nominal_8TBs": traffic / (fused_ms * 1e-3) / 1e9 / 8000.0},
+        "floor": {"bytes": 12.0 * d + 12.0 * nnz_mean,
+                  "note": "read g and eps once, write u once, the pairs and the cleared slots: what no "
+                          "implementation of the step can avoid moving",
+                  "gbs": (12.0 * d + 12.0 * nnz_mean) / (fused_ms * 1e-3) / 1e9,
+                  "frac_of_measured_copy": (12.0 * d + 12.0 * nnz_mean) / (fused_ms * 1e-3) / 1e9 / peak,
+                  "frac_of_nominal_8TBs": (12.0 * d + 12.0 * nnz_mean) / (fused_ms * 1e-3) / 1e9 / 8000.0},
     }
     # the three-kernel path (look-back compaction) on the same steps, stage by stage
     gk.gk_set_path(1)
@@ -397,6 +468,10 @@ def run_ours(args):
         topk[name] = rec
     gk.gk_set_path(0)
     ms_topk, ms_topk_sp = topk["fused"]["topk_exact_ms"], topk["fused"]["topk_sparsify_ms"]
+    # Gaussian_k as an operator on the same given vectors (Fig. 4 compares the operators)
+    for t in range(3):
+        gk.gk_select(us[t % len(us)], k, idx, val, nnz)
+    ms_gk_op = time_region(torch, lambda t: gk.gk_select(us[t % len(us)], k, idx, val, nnz), Kt) / Kt
 
     # ---- DGC_k (the paper's third operator, Section 4.3: a 1 % sample) on the same data, as
     # operator and as sparsifier; a fresh seeded sample per step, resident on the device
@@ -427,6 +502,7 @@ def run_ours(args):
             "dgck_select_gbs_4B_per_elem": (4.0 * d + 32.0 * m_s + 8.0 * k) / ms_dg_op / 1e6,
             "dgck_sparsify_gbs_12B_per_elem": (12.0 * d + 64.0 * m_s + 12.0 * k) / ms_dg_sp / 1e6,
             "vs_gaussiank_sparsify": ms_dg_sp / (ms / K), "vs_topk_sparsify": ms_dg_sp / ms_topk_sp,
+            "vs_gaussiank_select": ms_dg_op / ms_gk_op, "vs_topk_exact": ms_dg_op / ms_topk,
             "candidates_last": dg_info[1], "k_m": dg_info[2], "pairs_last": dg_info[3],
             "phase_ms_operator": dict(zip(dg_names, (acc_op / 20).tolist())),
             "phase_ms_sparsifier": dict(zip(dg_names, (acc_sp / 20).tolist())),
@@ -547,15 +623,23 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "repeats": len(regions), "steps_per_s": K / (ms * 1e-3) * world,
+        "gbs_at_20_bytes_per_element": whole_job_gbs(world, algorithmic_bytes(d, nnz_mean, 1.0), K, ms),
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": f"{w.name} d={d} rho={rho} k={k} whole-vector selection, eps carried over",
+            "workload": workload_string(w, rho),
             "l2": f"inputs per step g+eps = {8 * d / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2; "
                   f"{n_rot} gradient and {n_eps} residual buffers in rotation "
                   f"(episodes of {EPISODE} steps from eps = 0); no flush in the headline loop",
             "path": "fused cooperative kernel (1 launch per step)",
             "bytes_per_step": bytes_step, "nnz_last_step": nnz_mean,
+            "bytes_model": f"(16 + 4 r) d + 12 nnz, r = {r_passes:g} count passes over u in the last step",
+            "counting": {"ctas": info[4], "ctas_with_prediction": info[0], "ctas_whose_bands_held": info[1],
+                         "second_full_count": info[2], "cells_left_to_second_phase": info[3],
+                         "cells": (d // 4096) * 32},
+            "timed": f"{len(regions)} repeats of the {K}-step region, median reported "
+                     f"(min {min(regions) / K * 1e3:.2f} us, max {max(regions) / K * 1e3:.2f} us per step)",
             "parallelism": "replicas only" if world > 1 else "single GPU",
         },
         "pct_of_hbm_peak": {"measured_copy": value / world / peak, "nominal_8TBs": value / world / 8000.0},
@@ -563,9 +647,11 @@ def run_ours(args):
         "roofline": roof, "three_kernel_path": three,
         "cold_l2": {"ms_per_step": statistics.median(cold), "gbs": bytes_step / statistics.median(cold) / 1e6,
                     "note": "256 MB written between steps; per-step CUDA events"},
-        "topk": {"topk_exact_ms": ms_topk, "topk_sparsify_ms": ms_topk_sp,
-                 "speedup_operator_vs_sparsifier": ms_topk / (ms / K),
+        "topk": {"topk_exact_ms": ms_topk, "topk_sparsify_ms": ms_topk_sp, "gaussiank_select_ms": ms_gk_op,
+                 "speedup_operator": ms_topk / ms_gk_op,
                  "speedup_sparsifier": ms_topk_sp / (ms / K),
+                 "note": "operator against operator (gk_select vs topk_exact on a given u, the comparison of "
+                         "Fig. 4) and sparsifier against sparsifier (gk_sparsify vs topk_sparsify)",
                  "fused": topk["fused"], "multi_kernel": topk["multi_kernel"],
                  "paper_context": "paper: exact Top_k 0.4 s at this d on one V100 (Section 3.3)"},
         "segmented": seg, "dgck": dgck, "update_from_messages": upd, "diagnostics": diag, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": int(launches),
@@ -638,6 +724,10 @@ def run_sweep(args):
                 rec["segmented_ms"] = ms_seg
                 rec["segmented_gbs"] = algorithmic_bytes(d, int(nnz.item())) / ms_seg / 1e6
             u = gs[0]
+            for _ in range(3):
+                gk.gk_select(u, k, idx, val, nnz)
+            ms_gko = time_region(torch, lambda t: gk.gk_select(u, k, idx, val, nnz), 10) / 10
+            rec["gaussiank_select_ms"] = ms_gko
             tk_i = torch.empty(k, dtype=torch.int32, device=dev)
             tk_v = torch.empty(k, dtype=torch.float32, device=dev)
             for _ in range(3):
@@ -651,6 +741,7 @@ def run_sweep(args):
             ms_dgs = timed(lambda t: gk.dgck_sparsify(gs[t % n_grad], eps, k, smp, tk_i, tk_v, nnz))
             rec.update({"topk_exact_ms": ms_tk, "topk_sparsify_ms": ms_tks,
                         "speedup_vs_topk_sparsify": ms_tks / ms_gk,
+                        "speedup_select_vs_topk_exact": ms_tk / ms_gko,
                         "topk_exact_gbs_12B_per_elem": 12.0 * d / ms_tk / 1e6,
                         "dgck_select_ms": ms_dg, "dgck_sparsify_ms": ms_dgs,
                         "dgck_candidates_last": gk.dgck_last_info()[1]})
@@ -672,7 +763,7 @@ def main():
                     help="number of gradient buffers kept on the device (default 20; small for captures)")
     ap.add_argument("--loop-only", action="store_true",
                     help="run only warm-up and the timed loop (for profiler captures)")
-    ap.add_argument("--call", default="gk", choices=["gk", "segmented", "topk_exact", "topk_sparsify", "dgck_select", "dgck_sparsify"],
+    ap.add_argument("--call", default="gk", choices=["gk", "gk_select", "segmented", "topk_exact", "topk_sparsify", "dgck_select", "dgck_sparsify"],
                     help="entry point the timed loop calls (other than gk: with --loop-only, for captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every workload family (Gaussian_k, segmented, exact Top_k) and print one line each")

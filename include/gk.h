@@ -99,6 +99,24 @@ int gk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_o
                 float* val_out, int64_t* nnz_out, gk_stream_t stream);
 
 /*
+ * gk_select -- Gaussian_k as an operator on a given vector (Algorithm 1 of the paper as
+ * printed: input u, output the entries with |u_i| > threshold).  The same statistics,
+ * first threshold, count-and-adjust rounds and returned mask as gk_sparsify, without the
+ * accumulation before and the residual after: this is the form whose running time
+ * Section 4.3 / Fig. 4 compares with Top_k and DGC_k (topk_exact and dgck_select here).
+ *
+ *   u        DEVICE in   d floats, not modified (16-byte aligned)
+ *   d, k     sizes, 1 <= k <= d
+ *   idx_out  DEVICE out  capacity ints (gk_set_capacity; default d), ascending positions
+ *   val_out  DEVICE out  capacity floats: u at those positions
+ *   nnz_out  DEVICE out  one int64: number of pairs written
+ * Capacity rule, statistics record (gk_last_stats) and the choice of implementation
+ * (gk_set_path) as for gk_sparsify.
+ */
+int gk_select(const float* u, int64_t d, int64_t k, int32_t* idx_out, float* val_out,
+              int64_t* nnz_out, gk_stream_t stream);
+
+/*
  * gk_sparsify_segmented -- the same step with Algorithm 1 run independently on
  * every contiguous segment [seg_offsets[s], seg_offsets[s+1]) with its own
  * mean, deviation, k_s and threshold (layer-wise selection).  The paper states
@@ -335,6 +353,36 @@ int gk_last_stage_ms(gk_stream_t stream, float* ms_out, int* n_stages);
  * *n_ctas receives the number of CTAs, 0 if the last call did not run such a kernel.
  */
 int gk_last_cta_trace(gk_stream_t stream, uint64_t* host_out, int* n_ctas);
+
+/*
+ * gk_debug_set -- test hooks (the paper has no counterpart).  They exist so that tests can
+ * reach the give-up branch of every bounded wait without hanging anything, and both sides of
+ * the library's run-time decisions.  Process-wide; the device-side values are set on the
+ * current device.  Defaults are restored by setting the default value again.
+ *   key 0  polls of a grid barrier before a CTA gives up and sets GK_DEV_TIMEOUT (default 2^24)
+ *   key 1  polls of a predecessor's status word in the look-back compaction (default 2^22)
+ *   key 2  arrivals the barriers of the fused gk_sparsify kernel wait for beyond the grid
+ *          size (default 0).  With 1 no barrier can complete: every CTA's wait runs out,
+ *          the call ends with GK_DEV_TIMEOUT in gk_stats.status and invalid outputs.
+ *   key 3  a tile of the look-back compaction that keeps its status word to itself, so
+ *          that its successors' waits run out (default -1: none)
+ *   key 4  counting against predicted thresholds in the fused gk_sparsify / gk_select
+ *          kernel: -1 automatic (large vectors), 0 never, 1 whenever the vector has 128
+ *          elements or more
+ * Returns GK_ERR_SIZE for an unknown key or a value outside [-1, 2^31 - 1].
+ */
+int gk_debug_set(int key, int64_t value);
+
+/*
+ * How the last single-kernel gk_sparsify / gk_select call on `stream` took its counts
+ * (tracing aid).  Synchronises the stream and writes 5 int64 to HOST host_out: CTAs that
+ * formed a prediction of the thresholds from the sample; CTAs whose predicted bands held the
+ * exact thresholds (their counts come from the first phase plus the cells it left over);
+ * 1 if the rounds needed a candidate the short way leaves out, so that a full count followed;
+ * (row, warp) cells of 128 elements left to the second phase by CTAs with a prediction; CTAs
+ * of the launch (0 if the call did not run that kernel).
+ */
+int gk_last_path_info(gk_stream_t stream, int64_t* host_out);
 
 /* Number of kernels the library has launched so far in this process. */
 int64_t gk_launch_count(void);

@@ -26,7 +26,7 @@ EXPORTS = [
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
     "gk_error_ratio", "dgck_select", "dgck_sparsify", "dgck_last_info",
-    "gk_apply_sparse", "gk_apply_gathered", "gk_histogram",
+    "gk_apply_sparse", "gk_apply_gathered", "gk_histogram", "gk_debug_set", "gk_last_path_info", "gk_select",
 ]
 
 
@@ -75,6 +75,8 @@ def load() -> C.CDLL:
     L = C.CDLL(LIB_PATH)
     vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int32
     L.gk_sparsify.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.gk_select.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+    L.gk_select.restype = C.c_int
     L.gk_sparsify_static.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     L.gk_sparsify_static.restype = C.c_int
     L.gk_error_ratio.argtypes = [vp, i64, vp, vp, vp, C.POINTER(C.c_double)]
@@ -115,6 +117,10 @@ def load() -> C.CDLL:
     L.gk_last_cuda_error.argtypes = []
     L.gk_last_cuda_error.restype = C.c_char_p
     L.gk_version.argtypes = []
+    L.gk_last_path_info.argtypes = [vp, C.POINTER(i64)]
+    L.gk_last_path_info.restype = C.c_int
+    L.gk_debug_set.argtypes = [C.c_int, i64]
+    L.gk_debug_set.restype = C.c_int
     for name in ("gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
                  "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_last_stats", "gk_last_segment_stats", "gk_version"):
         getattr(L, name).restype = C.c_int
@@ -152,6 +158,13 @@ def gk_sparsify(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
     _check(load().gk_sparsify(_dev(g, torch.float32), _dev(eps, torch.float32), d, k,
                               _dev(idx_out, torch.int32), _dev(val_out, torch.float32),
                               _dev(nnz_out, torch.int64), _stream()))
+
+
+def gk_select(u, k: int, idx_out, val_out, nnz_out) -> None:
+    """Gaussian_k as an operator on a given vector u, which is not modified (see gk.h)."""
+    import torch
+    _check(load().gk_select(_dev(u, torch.float32), u.numel(), k, _dev(idx_out, torch.int32),
+                            _dev(val_out, torch.float32), _dev(nnz_out, torch.int64), _stream()))
 
 
 def gk_sparsify_static(g, eps, k: int, idx_out, val_out, nnz_out) -> None:
@@ -311,6 +324,24 @@ def gk_last_cta_trace():
     n = C.c_int(0)
     _check(load().gk_last_cta_trace(_stream(), buf, C.byref(n)))
     return [tuple(int(buf[i * 8 + j]) for j in range(8)) for i in range(n.value)]
+
+
+KNOB_BARRIER_POLLS, KNOB_LOOKBACK_POLLS, KNOB_EXTRA_ARRIVALS, KNOB_MUTE_TILE, KNOB_PREDICTION = range(5)
+
+
+def gk_debug_set(key: int, value: int) -> None:
+    """Test hooks (see gk.h): poll limits of the bounded waits, and switches that force either
+    side of the library's run-time decisions."""
+    _check(load().gk_debug_set(key, value))
+
+
+def gk_last_path_info():
+    """(CTAs with a prediction, CTAs whose bands held, second count needed, cells left to the
+    second phase, CTAs launched) of the last fused gk_sparsify / gk_select call on the current
+    stream.  Synchronises the stream."""
+    out = (C.c_int64 * 5)()
+    _check(load().gk_last_path_info(_stream(), out))
+    return tuple(int(v) for v in out)
 
 
 def gk_launch_count() -> int:

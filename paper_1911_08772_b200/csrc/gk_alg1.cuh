@@ -109,12 +109,14 @@ __device__ inline void alg1_thresholds(const Alg1State& a, double s1, double s2,
 struct Alg1Path {
     int chosen;                  // candidate index of the returned mask
     int rounds;                  // rounds executed
+    unsigned int visited;        // bit ci set: candidate ci was evaluated in some round
     long long est[kMaxRounds];   // the count seen in each round
 };
 __device__ inline Alg1Path alg1_replay(const unsigned long long* counts, int64_t k) {
     Alg1Path p;
     p.chosen = 0;
     p.rounds = 0;
+    p.visited = 0u;
     int h = 0, b = 0;
     bool going = true;
     // four rounds at most, written out so that nothing is indexed by a run-time value (arrays
@@ -128,6 +130,7 @@ __device__ inline Alg1Path alg1_replay(const unsigned long long* counts, int64_t
             est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&counts[ci]);
             p.rounds = r + 1;
             p.chosen = ci;
+            p.visited |= 1u << ci;
             if (3 * est < 2 * k) ++h;       // thres <- 0.5 * thres
             else if (3 * est > 4 * k) ++b;  // thres <- 1.5 * thres
             else going = false;
@@ -146,11 +149,14 @@ __device__ inline long long alg1_last_est(const Alg1Path& p) {
 }
 
 // The same with the record filled in.  One thread.
-// Returns the index of the candidate whose mask is returned (-1: everything).
-__device__ inline int alg1_resolve(const Alg1State& a, int64_t k) {
+// Returns the index of the candidate whose mask is returned (-1: everything).  visited_out, when
+// given, receives the set of candidates the rounds evaluated (bit = candidate index).
+__device__ inline int alg1_resolve(const Alg1State& a, int64_t k, unsigned int* visited_out = nullptr) {
     gk_stats* st = a.stats;
+    if (visited_out) *visited_out = 0u;
     if (st->rounds == 0 && st->thr_final == -INFINITY) return -1;  // everything selected
     const Alg1Path p = alg1_replay(a.counts, k);
+    if (visited_out) *visited_out = p.visited;
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) st->counts[r] = p.est[r];   // rounds not run keep 0
     st->rounds = p.rounds;

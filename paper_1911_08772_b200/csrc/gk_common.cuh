@@ -33,6 +33,21 @@ constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction 
 // Bounded waits: polls of a predecessor's status word before giving up.
 constexpr int kLookbackPollLimit = 1 << 22;
 
+// Test hooks (gk_debug_set): knobs that let a test reach the give-up branches of the bounded
+// waits and both sides of run-time decisions.  The device-side ones live in one variable per
+// translation unit (no relocatable device code); each unit registers a setter for its copy.
+enum Knob {
+    kKnobBarrierPolls = 0,    // polls of a grid barrier before a CTA gives up
+    kKnobLookbackPolls = 1,   // polls of a predecessor's status word before a tile gives up
+    kKnobExtraArrivals = 2,   // host: arrivals the fused kernels' barriers expect beyond the grid size
+    kKnobMuteTile = 3,        // compaction tile that does not publish its status word (-1: none)
+    kKnobPrediction = 4,      // host: -1 automatic, 0 never, 1 whenever possible (gk_fused.cu)
+    kKnobCount = 5
+};
+typedef int (*KnobSetter)(int key, int value);   // returns a cudaError_t as int
+int register_knob_setter(KnobSetter fn);
+int host_knob(int key);
+
 // Tile status word of the decoupled look-back: flag in bits 63..62, payload below.
 constexpr unsigned long long kFlagShift = 62;
 constexpr unsigned long long kFlagAggregate = 1ull;
@@ -61,6 +76,10 @@ struct Ctrl {
     // thresholds, after its counting loop, after the second barrier, after the replay of the
     // rounds, at the end of its compaction; and of the CTA that leaves last
     unsigned long long phase_t[8];
+    // fused Gaussian_k kernel, how the last call counted: CTAs that formed a prediction, CTAs whose
+    // predicted bands held the exact thresholds, whether a second full count was needed, cells
+    // left to phase B by CTAs with a prediction
+    unsigned int path_info[4];
     // gk_error_ratio: ratio, ||u - Comp(u)||^2, ||u||^2
     double diag[4];
     // DGC_k: key of the sampled threshold, candidates at or above it, rank taken in the sample,
@@ -77,8 +96,8 @@ struct Workspace {
     double2* partials = nullptr;            // kMaxPartials
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
-    unsigned int* cta_counts = nullptr;     // fused kernel: kFusedGridCap x kNumCand
-    unsigned int* bars = nullptr;           // 16 counters: [0..3] fused sparsifier, [4..8] fused Top_k, [10..13] fused segmented
+    unsigned int* cta_counts = nullptr;     // DGC_k and segmented fused kernels: per-CTA words (kFusedGridCap x kNumCand)
+    unsigned int* bars = nullptr;           // 64 words: [0..3], [9], [14..35] fused sparsifier, [4..8] fused Top_k, [10..13] fused segmented
     unsigned int* rowcnt = nullptr;         // fused kernels: two words per row of 4096 elements
     unsigned long long* cta_trace = nullptr;  // fused kernel: kFusedGridCap x 8 timestamps (tracing aid)
     int last_grid = 0;                      // CTAs of the last fused launch
@@ -100,7 +119,8 @@ void note_launch(int n = 1);
 void stage_mark(Workspace* ws, cudaStream_t st, int i);
 int64_t output_capacity(int64_t d);
 int selected_path();  // 0: fused kernel when usable, 1: three kernels with look-back
-int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+// eps == nullptr: the operator on a given vector (src = u, read only)
+int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                      float* val_out, int64_t* nnz_out, cudaStream_t st);
 int enqueue_topk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                        float* val_out, int64_t* nnz_out, cudaStream_t st);

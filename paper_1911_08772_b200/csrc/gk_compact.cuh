@@ -77,6 +77,17 @@ __device__ __forceinline__ unsigned int tile_scan(const unsigned int (&c)[kCompa
 // 31-bit counts, whose sums never carry into each other because d < 2^31).  Called by all
 // threads; returns to all of them the sum of the payloads of all earlier tiles, and
 // publishes this tile's inclusive prefix.
+// Test hooks of this translation unit: the poll limit of the look-back, and a tile that keeps
+// its status word to itself (-1: none), which makes its successors' bounded waits run out.
+static __device__ int g_lookback_poll_limit = kLookbackPollLimit;
+static __device__ int g_lookback_mute_tile = -1;
+static int set_compact_knob(int key, int value) {
+    if (key == kKnobLookbackPolls) return (int)cudaMemcpyToSymbol(g_lookback_poll_limit, &value, sizeof(int));
+    if (key == kKnobMuteTile) return (int)cudaMemcpyToSymbol(g_lookback_mute_tile, &value, sizeof(int));
+    return 0;
+}
+static const int g_compact_knob_registered = register_knob_setter(&set_compact_knob);
+
 struct LookbackSmem {
     unsigned long long sum_all[kCompactThreads / 32];
     unsigned long long sum_upto[kCompactThreads / 32];
@@ -90,12 +101,14 @@ __device__ __forceinline__ unsigned long long lookback_block(unsigned long long*
                                                              LookbackSmem& sm) {
     constexpr int NW = kCompactThreads / 32;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const bool mute = (tile == g_lookback_mute_tile);
+    const int poll_limit = g_lookback_poll_limit;
     if (tile == 0) {
-        if (tid == 0) st_status(&status[0], (kFlagPrefix << kFlagShift) | aggregate);
+        if (tid == 0 && !mute) st_status(&status[0], (kFlagPrefix << kFlagShift) | aggregate);
         return 0ull;
     }
     if (tid == 0) {
-        st_status(&status[tile], (kFlagAggregate << kFlagShift) | aggregate);
+        if (!mute) st_status(&status[tile], (kFlagAggregate << kFlagShift) | aggregate);
         sm.gave_up = 0;
     }
     __syncthreads();
@@ -107,7 +120,7 @@ __device__ __forceinline__ unsigned long long lookback_block(unsigned long long*
         unsigned long long wd = (mine >= 0) ? ld_status(&status[mine]) : (kFlagPrefix << kFlagShift);
         int polls = 0;
         while ((wd >> kFlagShift) == 0ull) {  // bounded wait for this predecessor's word
-            if (++polls > kLookbackPollLimit) { sm.gave_up = 1; break; }
+            if (++polls > poll_limit) { sm.gave_up = 1; break; }
             __nanosleep(20);
             wd = ld_status(&status[mine]);
         }
@@ -142,7 +155,7 @@ __device__ __forceinline__ unsigned long long lookback_block(unsigned long long*
         if (tid == 0) atomicOr(dev_status, GK_DEV_TIMEOUT);
         excl = 0ull;
     }
-    if (tid == 0) st_status(&status[tile], (kFlagPrefix << kFlagShift) | (excl + aggregate));
+    if (tid == 0 && !mute) st_status(&status[tile], (kFlagPrefix << kFlagShift) | (excl + aggregate));
     return excl;
 }
 

@@ -34,9 +34,10 @@ __device__ __forceinline__ int find_segment(const int64_t* __restrict__ off, int
 }
 
 // ---------------------------------------------------------------------------
-// Kernel C.  Survivors |u_i| > thr_sel -> ordered pairs; eps slot cleared.
+// Kernel C.  Survivors |u_i| > thr_sel -> ordered pairs; eps slot cleared (CLEAR; the
+// operator form leaves the vector as it is).
 // ---------------------------------------------------------------------------
-template <bool SEG>
+template <bool SEG, bool CLEAR = true>
 __global__ void __launch_bounds__(kCompactThreads)
 k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
                     unsigned long long* __restrict__ tile_status, int n_tiles,
@@ -149,7 +150,7 @@ k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
                         if ((int64_t)pos < cap) {
                             idx_out[pos] = (int32_t)(e0 + t);
                             val_out[pos] = vv[t];
-                            u[e0 + t] = 0.0f;
+                            if (CLEAR) u[e0 + t] = 0.0f;
                         }
                         ++pos;
                     }
@@ -164,7 +165,7 @@ k_compact_threshold(float* __restrict__ u, int64_t d, Ctrl* __restrict__ ctrl,
                 if ((int64_t)pos < cap) {
                     idx_out[pos] = (int32_t)((n4 << 2) + t);
                     val_out[pos] = tailv[t];
-                    u[(n4 << 2) + t] = 0.0f;
+                    if (CLEAR) u[(n4 << 2) + t] = 0.0f;
                 }
                 ++pos;
             }

@@ -15,6 +15,14 @@ constexpr int kBarrierPollLimit = 1 << 24;
 
 #ifdef __CUDACC__
 
+// Poll limit of grid_barrier in this translation unit (a test may lower it).
+static __device__ int g_barrier_poll_limit = kBarrierPollLimit;
+static int set_coop_knob(int key, int value) {
+    if (key != kKnobBarrierPolls) return 0;
+    return (int)cudaMemcpyToSymbol(g_barrier_poll_limit, &value, sizeof(int));
+}
+static const int g_coop_knob_registered = register_knob_setter(&set_coop_knob);
+
 // 16-byte asynchronous copy global -> shared, bypassing L1.
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
     const unsigned int s = (unsigned int)__cvta_generic_to_shared(smem);
@@ -39,12 +47,13 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
         __threadfence();
         atomicAdd(counter, 1u);
         int polls = 0;
+        const int limit = g_barrier_poll_limit;
         bool ok = true;
         while (true) {
             unsigned int v;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
             if (v >= G) break;
-            if (++polls > kBarrierPollLimit) { ok = false; break; }
+            if (++polls > limit) { ok = false; break; }
             __nanosleep(40);
         }
         *ok_flag = ok ? 1 : 0;

@@ -1,5 +1,5 @@
-// gk_sparsify as ONE persistent cooperative kernel (Eq. 2 and Algorithm 1 of
-// arXiv 1911.08772).
+// gk_sparsify (and gk_select, the same selection on a given u) as ONE persistent
+// cooperative kernel (Eq. 2 and Algorithm 1 of arXiv 1911.08772).
 //
 // The vector is cut into rows of 1024 float4 (16 KB; thread t takes float4 t of
 // the row), dealt to one CTA per SM in turn (CTA c owns rows c, c + G, ...), so
@@ -11,23 +11,45 @@
 //            kStages - 1 rows ahead); u = g + eps is written over eps and into the
 //            shared-memory slot its eps came through, so the last rows of the
 //            run are still on chip afterwards; fp64 partial sums per CTA; per
-//            (row, warp) the largest magnitude goes to a small table.
+//            (row, warp) cell the largest magnitude goes to a small table.
+//            On large vectors most of the counting of Algorithm 1 happens here
+//            as well, against PREDICTED thresholds (below).
 //   barrier  every CTA adds the partials in the same fixed order and forms
 //            mu, sigma, thres0 and the ten candidate thresholds for itself.
-//   phase B  counts of |u| > candidate for all ten candidates, from the
-//            on-chip copy where there is one, else from eps (L2 / HBM).
-//   barrier  every CTA reads all CTAs' counts and replays the rounds of
-//            Algorithm 1: threshold and number of survivors are known.
-//   phase C  a (row, warp) segment is read again only if its recorded maximum
-//            can exceed the threshold; the survivors of every row are counted
-//            and the counts exchanged through a third barrier, which gives
-//            every row its output offset -- no look-back, no waiting between
-//            CTAs; the survivors are written as (index, value) pairs and
-//            their slots cleared.
+//   phase B  counts of |u| > candidate, from the on-chip copy where there is
+//            one, else from eps (L2 / HBM): for all ten candidates over all
+//            cells, or, when the prediction held, for the six upper candidates
+//            over the cells that phase A could not settle.
+//   barrier  the CTAs' counts meet in ten global sums; every CTA replays the
+//            rounds of Algorithm 1: threshold and number of survivors are known.
+//   phase C  a cell is read again only if its recorded maximum can exceed the
+//            threshold; the survivors of every row are counted and the counts
+//            exchanged through a third barrier, which gives every row its output
+//            offset -- no look-back, no waiting between CTAs; the survivors are
+//            written as (index, value) pairs and their slots cleared.
 //
-// HBM traffic: 12 d bytes for phase A, 4 d for phase B on the rows that are not
-// on chip, and next to nothing for phase C (survivors are rare, so few segments
-// qualify).
+// Counting while the vector streams in.  The thresholds depend on mu and sigma
+// of the whole vector, which are known only after phase A.  But they can be
+// predicted: every warp first reads one block of 128 elements (the blocks of
+// all warps of all CTAs are spread evenly over the vector: a systematic sample
+// of about 1/42 of it at the benchmark size), the CTAs publish the sample's
+// power sums, and a few rows later every CTA forms a predicted first threshold
+// with an error bound delta from the sample's own fourth moment.  From then on
+// phase A counts, for each of the six candidates thres0 * {3/4, 1, 9/8, 3/2,
+// 9/4, 27/8}, the elements above hi_j = c_j (1 + delta), and notes for every
+// cell whether any element lies in a band (lo_j, hi_j].  A cell without such an
+// element has the same count for every threshold inside the band, so once the
+// exact c_j is known to lie in its band the phase A count of that cell is the
+// exact one; cells with a band element ("flagged"), rows that streamed before
+// the prediction arrived, and CTAs whose band missed are counted in phase B as
+// before.  The four lower candidates (thres0 / 8 ... thres0 / 2) are reached
+// only when the first count is below 2k/3; then every CTA that took the short
+// way counts again in full and one more barrier follows.  The result is exact
+// in every case: prediction only decides where a cell is counted.
+//
+// HBM traffic: 12 d bytes for phase A (4 d for gk_select), phase B's re-reads
+// (L2 mostly), and next to nothing for phase C (survivors are rare, so few
+// cells qualify).
 //
 // The barriers are counters in the workspace.  Every wait is bounded; a CTA
 // whose wait runs out records GK_DEV_TIMEOUT and leaves.  The kernel is
@@ -55,6 +77,36 @@ constexpr int kTraceSlots = 8;                         // timestamps per CTA in 
 // segment: one word each) in the ring's shared memory between counting and write-out
 constexpr int kStageCap = kRing * kRowF4 * 4;
 
+// Counting during phase A (prediction of the thresholds from a sample).
+constexpr int kUpper = 6;               // candidates thres0 * {3/4, 1, 9/8, 3/2, 9/4, 27/8}: sorted places 4..9
+constexpr int kPredMinRows = 10;        // rows per CTA from which on the prediction is tried
+constexpr int kPredPollFirst = 2;       // first row before which a CTA looks for the sample totals
+constexpr int kSampleElems = kFusedThreads * 4;   // sample elements per CTA: one float4 per thread
+constexpr double kPredSigmas = 3.5;     // half width of the bands in standard errors of the predicted threshold
+constexpr double kPredSlack = 5e-4;     // added to the relative half width
+constexpr double kPredMaxDelta = 0.05;  // wider bands than this are not worth counting against
+constexpr unsigned int kFlagBit = 0x8000u;   // table entry: the cell was not settled in phase A
+constexpr unsigned int kMaxMask = 0x7fffu;   // table entry: the cell's maximum (top 16 bits, rounded up)
+// candidates that only phase B's full count covers
+constexpr unsigned int kLowCandMask = (1u << cand_index(1, 0)) | (1u << cand_index(2, 0)) |
+                                      (1u << cand_index(3, 0)) | (1u << cand_index(2, 1));
+static_assert(cand_by_factor(0) == cand_index(3, 0) && cand_by_factor(1) == cand_index(2, 0) &&
+              cand_by_factor(2) == cand_index(2, 1) && cand_by_factor(3) == cand_index(1, 0),
+              "the four lowest factors are the candidates of kLowCandMask");
+
+// Words of the barrier block used by this kernel (the exact Top_k kernel has 4..8, the segmented
+// one 10..13).  All are zero between calls: the CTA that leaves last clears them.
+constexpr int kBarStats = 0;      // barrier after phase A
+constexpr int kBarCounts = 1;     // barrier after phase B
+constexpr int kBarExit = 2;       // CTAs that have left
+constexpr int kBarRows = 3;       // barrier inside phase C
+constexpr int kBarPublished = 9;  // CTAs whose sample sums are in place
+constexpr int kBarInvalid = 14;   // candidates (bit = index) that some CTA has not counted
+constexpr int kBarCounts2 = 15;   // barrier after the second, full count
+constexpr int kBarTotals = 16;    // 2 x kNumCand words: the global counts of the first and the second count
+constexpr int kBarInfo = 36;      // 4 words: what Ctrl::path_info reports, collected during the call
+constexpr int kBarWords = 64;
+
 struct __align__(128) FusedShared {
     double2 red[kFusedWarps];
     unsigned int cta_counts[kNumCand];
@@ -62,9 +114,14 @@ struct __align__(128) FusedShared {
     double cand64[kNumCand];
     float cand32[kNumCand];
     int order[kNumCand];                // candidate indices, ascending by threshold
+    float plo[kUpper], phi[kUpper];     // predicted bands of the six upper candidates
     float thr_sel;
     int chosen;
     int ok;
+    int poll[2];                        // the sample totals were complete when row r (parity) began
+    int pred_ok;                        // a usable prediction was formed
+    int fast;                           // this CTA's bands hold the exact candidates
+    int recount;                        // the rounds need a candidate that some CTA has not counted
     gk_stats stats;
     unsigned int wsum[kFusedWarps];
     unsigned int roundtot[kTableMaxRows];  // survivors in each round of rows (G consecutive rows)
@@ -81,19 +138,57 @@ __device__ __forceinline__ unsigned int mask_above(const float4 v, const float t
            ((unsigned)(fabsf(v.z) > thr) << 2) | ((unsigned)(fabsf(v.w) > thr) << 3);
 }
 
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// The predicted first threshold and its bands, from the sample's power sums about the pivot pv
+// (n sample elements).  The half width is kPredSigmas standard errors of mu + sigma z, with the
+// standard error of sigma taken from the sample's own fourth moment (heavy tails widen the
+// bands by themselves), plus a small slack.  Returns false when no useful prediction exists.
+__device__ inline bool predict_bands(double s1, double s2, double s3, double s4, double n, double pv, double z,
+                                     float* plo, float* phi) {
+    const double m1 = s1 / n, r2 = s2 / n, r3 = s3 / n, r4 = s4 / n;
+    const double var_p = r2 - m1 * m1;                    // population variance of the sample
+    if (!(var_p > 0.0) || !(n > 2.0)) return false;
+    const double var = var_p * n / (n - 1.0);
+    const double c4 = r4 - 4.0 * m1 * r3 + 6.0 * m1 * m1 * r2 - 3.0 * m1 * m1 * m1 * m1;   // central fourth moment
+    const double kurt = c4 / (var_p * var_p);
+    const double sigma = sqrt(var);
+    const double th = (pv + m1) + sigma * z;
+    if (!(th > 0.0) || !(th < 3.0e38)) return false;
+    const double se_sigma = 0.5 * sqrt(fmax(kurt - 1.0, 0.0) / n) * sigma;   // standard error of sigma
+    const double se_th = sqrt(var / n + z * z * se_sigma * se_sigma);
+    const double delta = kPredSigmas * se_th / th + kPredSlack;
+    if (!(delta < kPredMaxDelta)) return false;
+    const double f[kUpper] = {0.75, 1.0, 1.125, 1.5, 2.25, 3.375};
+#pragma unroll
+    for (int j = 0; j < kUpper; ++j) {
+        plo[j] = __double2float_rd(th * f[j] * (1.0 - delta));
+        phi[j] = __double2float_ru(th * f[j] * (1.0 + delta));
+    }
+    return phi[kUpper - 1] < 3.0e38f;
+}
+
+// ACC: the sparsifier (src = g, u = g + eps is formed, stored over eps and cleared where
+// selected); !ACC: the operator on a given vector (src = u, read only; eps is not used).
 // n_rows: rows of 1024 float4 in the whole vector; CTA c owns rows c, c + G, c + 2G, ...
 // (G = gridDim.x), so that stretches of large values are spread over all CTAs.  u_slots: row
 // slots of shared memory that receive eps and then hold u (the last u_slots rows of a CTA stay
 // on chip); table_rows: the largest number of rows any CTA owns (entries of the maximum table).
-// rowcnt: one word per row of the vector.
+// predict: count during phase A against predicted thresholds (the vector must have at least 32
+// float4); bar_target: arrivals a grid barrier waits for (the grid size; a test may ask for more
+// to see the bounded waits run out).  spart: two double2 per CTA.  rowcnt: one word per row.
 // Shared memory: [ring of kRing rows][u_slots rows][table of table_rows x 32 uint16].
+template <bool ACC>
 __global__ void __launch_bounds__(kFusedThreads, 1)
-k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
-           int n_rows, int u_slots, int table_rows, Ctrl* __restrict__ ctrl,
-           double2* __restrict__ partials, unsigned int* __restrict__ cta_counts,
-           unsigned int* __restrict__ bars, unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out,
-           float* __restrict__ val_out, int64_t* __restrict__ nnz_out, int64_t cap,
-           unsigned long long* __restrict__ trace) {
+k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, double z,
+           int n_rows, int u_slots, int table_rows, int predict, unsigned int bar_target, Ctrl* __restrict__ ctrl,
+           double2* __restrict__ partials, double2* __restrict__ spart, unsigned int* __restrict__ bars,
+           unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+           int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
     // 1 KB alignment keeps every warp's 512 bytes of a row within four 128-byte lines of shared
     // memory, whatever the size of the static part
     extern __shared__ __align__(1024) float4 smem4[];
@@ -117,10 +212,15 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     const int first_kept = nrows > u_slots ? nrows - u_slots : 0;
     const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
     const int64_t tail_i = (n4 << 2) + lane;
-    const float4* g4 = reinterpret_cast<const float4*>(g);
+    const float4* g4 = reinterpret_cast<const float4*>(src);
     float4* e4 = reinterpret_cast<float4*>(eps);
+    // where u is read again after phase A: eps holds it for the sparsifier, the input itself otherwise
+    const float* uvec = ACC ? eps : src;
+    const float4* u4 = reinterpret_cast<const float4*>(uvec);
     float tail_u = 0.f;
-    const bool wide_ok = ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
+    const bool wide_ok = ACC && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
+    unsigned int* tot0 = bars + kBarTotals;               // global counts of the first count
+    unsigned int* tot1 = bars + kBarTotals + kNumCand;    // ... of the second, full one
     if (c == 0 && tid == 0) {
         ctrl->stats.status = GK_DEV_OK;
         ctrl->phase_t[0] = global_timer_ns();
@@ -131,12 +231,20 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
     };
     stamp(0);
 
+    // phase A's counts of the six upper candidates over the cells it settled, and whether this
+    // CTA holds a prediction
+    float pacc[kUpper];
+#pragma unroll
+    for (int j = 0; j < kUpper; ++j) pacc[j] = 0.f;
+    bool pred_live = false;
+
     // ------------------------------------------------------------------ phase A
     {
-        const double pv = (double)g[0];
+        const double pv = (double)src[0];
         double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
         // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
         // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
+        // The operator form has one operand, which takes the way of eps.
         int64_t fi = first4;  // the row the next fetch brings in
         // Where the eps of local row r lands.  Normally the slot that will hold u.  A CTA with so
         // many rows that its table leaves fewer slots than rows in flight takes eps through the
@@ -147,26 +255,99 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
         };
         auto fetch = [&](int r) {
             if (r < nrows && fi < n4) {
-                cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
-                cp_async16(eps_slot(r) + tid, e4 + fi);
+                if (ACC) {
+                    cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
+                    cp_async16(eps_slot(r) + tid, e4 + fi);
+                } else {
+                    cp_async16(eps_slot(r) + tid, g4 + fi);
+                }
             }
             cp_async_commit();
             fi += stride4;
         };
 #pragma unroll
         for (int r = 0; r < kStages - 1; ++r) fetch(r);
+
+        // The sample: warp w of CTA c reads block (c * 32 + w) of G * 32 blocks of 32 float4 spread
+        // evenly over the vector, and the CTA publishes the power sums of (u - pv).  (Another CTA
+        // may already have replaced eps by u in a block of the first rows; the sample then sees
+        // g + u there.  That can only cost accuracy of the prediction, never of the result.)
+        int pred_state = 0;   // 1: sample published, totals not yet seen
+        if (predict) {
+            const int64_t nblk = n4 >> 5;
+            const int64_t blk = (((int64_t)c * kFusedWarps + w) * nblk) / ((int64_t)G * kFusedWarps);
+            const int64_t at = (blk << 5) + lane;
+            float4 a = __ldcg(g4 + at);
+            if (ACC) {
+                const float4 b = __ldcg(e4 + at);
+                a = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+            }
+            const double x[4] = {(double)a.x - pv, (double)a.y - pv, (double)a.z - pv, (double)a.w - pv};
+            double p1 = 0.0, p2 = 0.0, p3 = 0.0, p4 = 0.0;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const double y = x[t] * x[t];
+                p1 += x[t]; p2 += y; p3 = fma(y, x[t], p3); p4 = fma(y, y, p4);
+            }
+            const double2 a12 = block_sum2<kFusedThreads>(p1, p2, sh.red);
+            const double2 a34 = block_sum2<kFusedThreads>(p3, p4, sh.red);
+            if (tid == 0) {
+                spart[2 * c] = a12;
+                spart[2 * c + 1] = a34;
+                __threadfence();
+                atomicAdd(&bars[kBarPublished], 1u);
+            }
+            pred_state = 1;
+        }
+        unsigned int ptl0 = 0u, ptl1 = 0u, ptl3 = 0u;   // tier limits of the predicted bands
+        unsigned int n_left = 0u;                        // cells of this warp left to phase B
+        const int poll_end = nrows / 3;                  // a prediction that comes later is not worth having
+
         int64_t i = first4;
         for (int r = 0; r < nrows; ++r, i += stride4) {
+            if (pred_state == 1 && r >= kPredPollFirst) {
+                // have all CTAs published?  One look per row; the answer goes through shared memory
+                // (two words in turn, so that a thread still reading last row's cannot see this row's)
+                if (tid == 0) sh.poll[r & 1] = ld_acquire_u32(&bars[kBarPublished]) >= (unsigned)G ? 1 : 0;
+                __syncthreads();
+                if (sh.poll[r & 1]) {
+                    double a1 = 0.0, a2 = 0.0, a3 = 0.0, a4 = 0.0;
+                    for (int t = tid; t < G; t += kFusedThreads) {
+                        const double2 p = __ldcg(&spart[2 * t]), q = __ldcg(&spart[2 * t + 1]);
+                        a1 += p.x; a2 += p.y; a3 += q.x; a4 += q.y;
+                    }
+                    const double2 t12 = block_sum2<kFusedThreads>(a1, a2, sh.red);
+                    const double2 t34 = block_sum2<kFusedThreads>(a3, a4, sh.red);
+                    if (tid == 0)
+                        sh.pred_ok = predict_bands(t12.x, t12.y, t34.x, t34.y, (double)G * kSampleElems, pv, z,
+                                                   sh.plo, sh.phi) ? 1 : 0;
+                    __syncthreads();
+                    pred_state = 0;
+                    if (sh.pred_ok) {
+                        pred_live = true;
+                        // top 16 bits of each tier's lowest band edge, rounded down (the edges are positive)
+                        ptl0 = __float_as_uint(sh.plo[0]) >> 16;
+                        ptl1 = __float_as_uint(sh.plo[1]) >> 16;
+                        ptl3 = __float_as_uint(sh.plo[3]) >> 16;
+                    }
+                } else if (r >= poll_end) {
+                    pred_state = 0;
+                }
+            }
             fetch(r + kStages - 1);
             cp_async_wait<kStages - 1>();
             const bool one = i < n4;
             float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (one) {
                 float4* es = eps_slot(r) + tid;
-                const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *es;
-                u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
-                if (!eps_ring) *es = u0;
-                else if (r >= first_kept) uslot[(size_t)(r % u_slots) * kRowF4 + tid] = u0;
+                if (ACC) {
+                    const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *es;
+                    u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
+                    if (!eps_ring) *es = u0;
+                } else {
+                    u0 = *es;
+                }
+                if (eps_ring && r >= first_kept) uslot[(size_t)(r % u_slots) * kRowF4 + tid] = u0;
                 const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
                              x3 = (double)u0.w - pv;
                 s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
@@ -174,7 +355,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             }
             // u goes out in 32-byte stores by the even lanes (own float4 and the right neighbour's),
             // marked to stay in L2: the next two phases read most of u again
-            {
+            if (ACC) {
                 float4 nb;
                 nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
                 nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
@@ -186,29 +367,65 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                     e4[i] = u0;
                 }
             }
-            // largest magnitude of each (row, warp) segment, top 16 bits rounded up
+            // largest magnitude of each (row, warp) cell, top 16 bits rounded up (15 bits for
+            // finite values), and above it the flag "not settled here"
             const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
-            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)((m0 + 0xffffu) >> 16);
+            unsigned int entry = (m0 + 0xffffu) >> 16;
+            if (predict) {
+                if (!pred_live) {
+                    entry |= kFlagBit;
+                } else if (entry > ptl0) {
+                    // the cell can reach the lowest band: per candidate the elements above the band's
+                    // upper edge, and over all candidates those above the lower edges; the two sums
+                    // differ exactly when an element lies inside a band
+                    const float a0 = fabsf(u0.x), a1 = fabsf(u0.y), a2 = fabsf(u0.z), a3 = fabsf(u0.w);
+                    float h[kUpper];
+#pragma unroll
+                    for (int j = 0; j < kUpper; ++j) h[j] = 0.f;
+                    float below = 0.f;
+                    auto band = [&](const int j) {
+                        const float lo = sh.plo[j], hi = sh.phi[j];
+                        h[j] = (gt_as_float(a0, hi) + gt_as_float(a1, hi)) + (gt_as_float(a2, hi) + gt_as_float(a3, hi));
+                        below += (gt_as_float(a0, lo) + gt_as_float(a1, lo)) + (gt_as_float(a2, lo) + gt_as_float(a3, lo));
+                    };
+                    band(0);
+                    if (entry > ptl1) {
+                        band(1); band(2);
+                        if (entry > ptl3) { band(3); band(4); band(5); }
+                    }
+                    const float above = ((h[0] + h[1]) + (h[2] + h[3])) + (h[4] + h[5]);
+                    if (__any_sync(0xffffffffu, below != above)) {
+                        entry |= kFlagBit;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kUpper; ++j) pacc[j] += h[j];
+                    }
+                }
+            }
+            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)entry;
+            n_left += (entry >> 15);
         }
+        if (pred_live && lane == 0 && n_left) atomicAdd(&bars[kBarInfo + 3], n_left);
+        if (pred_live && tid == 0) atomicAdd(&bars[kBarInfo + 0], 1u);
         cp_async_wait<0>();
         if (owns_tail) {
-            tail_u = g[tail_i] + eps[tail_i];
-            eps[tail_i] = tail_u;
+            tail_u = ACC ? src[tail_i] + eps[tail_i] : src[tail_i];
+            if (ACC) eps[tail_i] = tail_u;
             const double x = (double)tail_u - pv;
             s0 += x; q0 = fma(x, x, q0);
         }
         const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
         if (tid == 0) partials[c] = part;
         stamp(1);
-        if (!grid_barrier(&bars[0], (unsigned)G, &sh.ok)) {
+        if (!grid_barrier(&bars[kBarStats], bar_target, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
         stamp(2);
         // every CTA forms the same totals: thread t takes partial t, t + T, ...
         double s = 0.0, q = 0.0;
-        for (int i = tid; i < G; i += kFusedThreads) {
-            const double2 p = __ldcg(&partials[i]);
+        for (int t = tid; t < G; t += kFusedThreads) {
+            const double2 p = __ldcg(&partials[t]);
             s += p.x; q += p.y;
         }
         const double2 tot = block_sum2<kFusedThreads>(s, q, sh.red);
@@ -219,121 +436,144 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             const bool neg = sh.stats.thres0 < 0.0;
 #pragma unroll
             for (int j = 0; j < kNumCand; ++j) sh.order[j] = cand_ascending(j, neg);
+            // phase A's counts stand if every exact candidate lies within its predicted band
+            bool fast = pred_live && sh.stats.thres0 > 0.0;
+            if (fast) {
+#pragma unroll
+                for (int j = 0; j < kUpper; ++j) {
+                    const float cj = sh.cand32[cand_by_factor(kNumCand - kUpper + j)];
+                    fast = fast && sh.plo[j] <= cj && cj <= sh.phi[j];
+                }
+            }
+            sh.fast = fast ? 1 : 0;
+            sh.recount = 0;
         }
         if (tid < kNumCand) sh.cta_counts[tid] = 0u;
         if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
         __syncthreads();
     }
 
-    // ------------------------------------------------------------------ phase B
-    {
-        // candidates in ascending order of value; cs[j] = value, sh.order[j] = its index
-        float cs[kNumCand], acc[kNumCand];
+    // ------------------------------------------------------------------ phase B and the rounds
+    // First count: the short way where this CTA's prediction held, else in full.  If the rounds
+    // then ask for a candidate that some CTA left out, the CTAs that took the short way count
+    // again in full and the sums are formed a second time.
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool fast = pass == 0 && sh.fast != 0;
+        if (pass == 0 || sh.fast != 0) {
+            // candidates in ascending order of value; cs[j] = value, sh.order[j] = its index
+            float cs[kNumCand], acc[kNumCand];
 #pragma unroll
-        for (int j = 0; j < kNumCand; ++j) { cs[j] = sh.cand32[sh.order[j]]; acc[j] = 0.f; }
-        // tier limits: top 16 bits of the tier's lowest candidate, rounded down; a negative
-        // candidate is exceeded by everything, and candidates ascend, so testing the lowest suffices
-        Tiers tier;
-        tier.t0 = __float_as_uint(fmaxf(cs[0], 0.f)) >> 16;
-        tier.t2 = __float_as_uint(fmaxf(cs[2], 0.f)) >> 16;
-        tier.t5 = __float_as_uint(fmaxf(cs[5], 0.f)) >> 16;
-        tier.t7 = __float_as_uint(fmaxf(cs[7], 0.f)) >> 16;
-        const unsigned int always = 0x10000u;  // above every 16-bit maximum
-        const bool any_neg = cs[0] < 0.f;
-        const unsigned short* trow = table + w;
-        // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
-        // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows.  They are
-        // taken from the last written to the first: the rows written last are the ones most
-        // likely still in L2, and reading them first keeps the misses on the oldest rows from
-        // pushing them out before their turn.
-        int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;  // the row the next fetch brings in
-        auto fetch_u = [&](int q) {   // q-th row in this order: local row first_kept - 1 - q
-            if (q < first_kept) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, e4 + fo);
-            cp_async_commit();
-            fo -= stride4;
-        };
-        auto row_max = [&](int r) -> unsigned int {
-            return any_neg ? always : (unsigned int)trow[r * kFusedWarps];
-        };
+            for (int j = 0; j < kNumCand; ++j) {
+                cs[j] = sh.cand32[sh.order[j]];
+                acc[j] = (fast && j >= kNumCand - kUpper) ? pacc[j - (kNumCand - kUpper)] : 0.f;
+            }
+            // tier limits: top 16 bits of the tier's lowest candidate, rounded down; a negative
+            // candidate is exceeded by everything, and candidates ascend, so testing the lowest suffices
+            Tiers tier = make_tiers(cs);
+            if (fast) tier.t0 = __float_as_uint(cs[kNumCand - kUpper]) >> 16;   // the short way starts at 3/4 thres0 (> 0)
+            const unsigned int always = 0x10000u;  // above every 16-bit maximum
+            const bool any_neg = cs[0] < 0.f;
+            const unsigned short* trow = table + w;
+            // is the cell of local row r to be counted now, and with which maximum
+            auto wanted = [&](int r) -> bool { return !fast || (trow[r * kFusedWarps] & kFlagBit) != 0u; };
+            auto row_max = [&](int r) -> unsigned int {
+                return any_neg ? always : ((unsigned int)trow[r * kFusedWarps] & kMaxMask);
+            };
+            auto count_cell = [&](const float4 x, const int r) {
+                if (fast) count_float4<kNumCand - kUpper>(x, row_max(r), cs, tier, acc);
+                else count_float4<0>(x, row_max(r), cs, tier, acc);
+            };
+            // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
+            // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows.  They are
+            // taken from the last written to the first: the rows written last are the ones most
+            // likely still in L2, and reading them first keeps the misses on the oldest rows from
+            // pushing them out before their turn.
+            int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;  // the row the next fetch brings in
+            auto fetch_u = [&](int q) {   // q-th row in this order: local row first_kept - 1 - q
+                if (q < first_kept && wanted(first_kept - 1 - q)) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, u4 + fo);
+                cp_async_commit();
+                fo -= stride4;
+            };
 #pragma unroll
-        for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
-        static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
-        int r = 0;
+            for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
+            static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
 #pragma unroll 2
-        for (int q = 0; q < first_kept; ++q) {
-            fetch_u(q + kRing - 1);
-            cp_async_wait<kRing - 1>();
-            count_float4(gring[((q & (kRing - 1)) << 10) + tid], row_max(first_kept - 1 - q), cs, tier, acc);
-        }
-        cp_async_wait<0>();
-        for (r = first_kept; r < nrows; ++r) {
-            if (r != nrows - 1 || in_last_row)
-                count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], row_max(r), cs, tier, acc);
-        }
-        if (owns_tail) {
-            const float a = fabsf(tail_u);
+            for (int q = 0; q < first_kept; ++q) {
+                fetch_u(q + kRing - 1);
+                cp_async_wait<kRing - 1>();
+                const int r = first_kept - 1 - q;
+                if (wanted(r)) count_cell(gring[((q & (kRing - 1)) << 10) + tid], r);
+            }
+            cp_async_wait<0>();
+            for (int r = first_kept; r < nrows; ++r) {
+                if ((r != nrows - 1 || in_last_row) && wanted(r))
+                    count_cell(uslot[(size_t)(r % u_slots) * kRowF4 + tid], r);
+            }
+            if (owns_tail) {
+                const float a = fabsf(tail_u);
 #pragma unroll
-            for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
-        }
+                for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
+            }
+            if (pass == 1) {
+                __syncthreads();   // the first count's sums have been read by everyone
+                if (tid < kNumCand) sh.cta_counts[tid] = 0u;
+                __syncthreads();
+            }
 #pragma unroll
-        for (int j = 0; j < kNumCand; ++j) {
-            const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
-            if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
+            for (int j = 0; j < kNumCand; ++j) {
+                const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+                if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        if (tid < kNumCand) cta_counts[(size_t)c * kNumCand + tid] = sh.cta_counts[tid];
+        // this CTA's counts join the global sums; the short way leaves the four lower candidates out
+        if (tid < kNumCand) {
+            const unsigned int v = sh.cta_counts[tid];
+            if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
+        }
+        if (fast && tid == 0) {
+            atomicOr(&bars[kBarInvalid], kLowCandMask);
+            atomicAdd(&bars[kBarInfo + 1], 1u);
+        }
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
         stamp(3);
-        if (!grid_barrier(&bars[1], (unsigned)G, &sh.ok)) {
+        if (!grid_barrier(&bars[pass == 0 ? kBarCounts : kBarCounts2], bar_target, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
         if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
         stamp(4);
-    }
 
-    // ------------------------------------------------------------------ resolve
-    {
-        // warp j adds column j over all CTAs (integer sums: the order does not matter); the loads
-        // are independent of each other
-        if (w < kNumCand) {
-            unsigned int v[kFusedMaxGrid / 32];
-#pragma unroll
-            for (int q = 0; q < kFusedMaxGrid / 32; ++q) {
-                const int t = lane + 32 * q;
-                v[q] = (t < G) ? __ldcg(&cta_counts[(size_t)t * kNumCand + w]) : 0u;
-            }
-            unsigned long long s = 0ull;
-#pragma unroll
-            for (int q = 0; q < kFusedMaxGrid / 32; ++q) s += v[q];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0) sh.col[w] = s;
-        }
+        // -------------------------------------------------------------- the rounds
+        if (tid < kNumCand) sh.col[tid] = (unsigned long long)ld_acquire_u32((pass == 0 ? tot0 : tot1) + tid);
         __syncthreads();
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
-            sh.chosen = alg1_resolve(st, k);
+            unsigned int visited = 0u;
+            sh.chosen = alg1_resolve(st, k, &visited);
             sh.n_staged = 0u;
+            // a candidate the rounds evaluated but some CTA did not count: count again, in full
+            sh.recount = (pass == 0 && (visited & ld_acquire_u32(&bars[kBarInvalid])) != 0u) ? 1 : 0;
         }
         __syncthreads();
-        if (c == 0 && tid == 0) {
-            const long long all = sh.stats.nnz;
-            const long long written = all < cap ? all : cap;
-            // every field but the status word, which was cleared at the start and only ever has
-            // flags added to it (a CTA that gave up waiting may have added one already)
-            gk_stats* o = &ctrl->stats;
-            o->mu = sh.stats.mu; o->sigma = sh.stats.sigma; o->z = sh.stats.z;
-            o->thres0 = sh.stats.thres0; o->thr_final = sh.stats.thr_final;
+        if (!sh.recount) break;
+        if (c == 0 && tid == 0) bars[kBarInfo + 2] = 1u;
+    }
+    if (c == 0 && tid == 0) {
+        const long long all = sh.stats.nnz;
+        const long long written = all < cap ? all : cap;
+        // every field but the status word, which was cleared at the start and only ever has
+        // flags added to it (a CTA that gave up waiting may have added one already)
+        gk_stats* o = &ctrl->stats;
+        o->mu = sh.stats.mu; o->sigma = sh.stats.sigma; o->z = sh.stats.z;
+        o->thres0 = sh.stats.thres0; o->thr_final = sh.stats.thr_final;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) o->counts[j] = sh.stats.counts[j];
-            o->rounds = sh.stats.rounds; o->nnz = all; o->emitted = written;
-            const int flags = sh.stats.status | (all > cap ? GK_DEV_TRUNCATED : 0);
-            if (flags) atomicOr(&o->status, flags);
-            *nnz_out = written;
-            ctrl->phase_t[4] = global_timer_ns();
-        }
-        __syncthreads();
+        for (int j = 0; j < 4; ++j) o->counts[j] = sh.stats.counts[j];
+        o->rounds = sh.stats.rounds; o->nnz = all; o->emitted = written;
+        const int flags = sh.stats.status | (all > cap ? GK_DEV_TRUNCATED : 0);
+        if (flags) atomicOr(&o->status, flags);
+        *nnz_out = written;
+        ctrl->phase_t[4] = global_timer_ns();
     }
 
     // ------------------------------------------------------------------ phase C
@@ -354,7 +594,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             while (n < kGroupRows && cursor < nrows) {
                 const int r = cursor + lane;
                 unsigned int e = 0u;
-                if (r < nrows) e = table[r * kFusedWarps + w];
+                if (r < nrows) e = table[r * kFusedWarps + w];   // a count by now, or the pending mark
                 const bool hit = want_pending ? (e == kPending) : (e != 0u);
                 unsigned int b = __ballot_sync(0xffffffffu, hit);
                 while (b && n < kGroupRows) {
@@ -370,7 +610,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             return n;
         };
         auto load_row = [&](int r, int64_t i) -> float4 {
-            return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);
+            return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(u4 + i);
         };
         // When this CTA's survivors fit the ring's shared memory (free since phase B), their
         // places -- row, warp, lane, element, rank within the segment: one word -- are put aside
@@ -384,7 +624,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             // entry of a segment is replaced by that count (0 where it cannot qualify).
             int pending = 0;
             for (int r = lane; r < nrows; r += 32) {
-                const bool ql = all_pass || table[r * kFusedWarps + w] > thr16;
+                const bool ql = all_pass || ((unsigned int)table[r * kFusedWarps + w] & kMaxMask) > thr16;
                 table[r * kFusedWarps + w] = ql ? kPending : (unsigned short)0;
                 pending += ql;
             }
@@ -494,7 +734,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
             rowcnt[c + tid * G] = mine_row;
         }
         stamp(5);
-        if (!grid_barrier(&bars[3], (unsigned)G, &sh.ok)) {
+        if (!grid_barrier(&bars[kBarRows], bar_target, &sh.ok)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
@@ -552,10 +792,10 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                         const int64_t at = (((int64_t)c + (int64_t)r * G) << 12) + in_row;
                         const float x = ((int)r >= first_kept)
                                             ? reinterpret_cast<const float*>(uslot + (size_t)(r % u_slots) * kRowF4)[in_row]
-                                            : __ldcg(eps + at);
+                                            : __ldcg(uvec + at);
                         idx_out[p] = (int32_t)at;
                         val_out[p] = x;
-                        eps[at] = 0.0f;
+                        if (ACC) eps[at] = 0.0f;
                     }
                 }
             } else
@@ -598,7 +838,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                                 if (p < cap) {
                                     idx_out[p] = (int32_t)(e0 + t);
                                     val_out[p] = vv[t];
-                                    eps[e0 + t] = 0.0f;
+                                    if (ACC) eps[e0 + t] = 0.0f;
                                 }
                                 ++p;
                             }
@@ -617,7 +857,7 @@ k_gk_fused(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int6
                 if (p < cap) {
                     idx_out[p] = (int32_t)tail_i;
                     val_out[p] = tail_u;
-                    eps[tail_i] = 0.0f;
+                    if (ACC) eps[tail_i] = 0.0f;
                 }
             }
         }
@@ -631,12 +871,15 @@ leave:
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        const unsigned int t = atomicAdd(&bars[2], 1u);
+        const unsigned int t = atomicAdd(&bars[kBarExit], 1u);
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[6] = global_timer_ns();
-            bars[0] = 0u; bars[1] = 0u; bars[3] = 0u;
+            bars[kBarStats] = 0u; bars[kBarCounts] = 0u; bars[kBarRows] = 0u;
+            bars[kBarPublished] = 0u; bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
+            for (int j = 0; j < 2 * kNumCand; ++j) bars[kBarTotals + j] = 0u;
+            for (int j = 0; j < 4; ++j) { ctrl->path_info[j] = bars[kBarInfo + j]; bars[kBarInfo + j] = 0u; }
             __threadfence();
-            bars[2] = 0u;
+            bars[kBarExit] = 0u;
         }
     }
 }
@@ -648,6 +891,22 @@ struct FusedPlan {
 };
 static FusedPlan g_plan[64];
 
+template <bool ACC>
+static bool fused_kernel_ready() {
+    if (cudaFuncSetAttribute(k_gk_fused<ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBudget) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused<ACC>, kFusedThreads, kFusedSmemBudget) !=
+            cudaSuccess || occ < 1) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
 static FusedPlan* fused_plan(int dev, int sm_count) {
     if (dev < 0 || dev >= 64) return nullptr;
     // built once per device, under a lock: a second thread's first call waits for the finished plan
@@ -658,17 +917,7 @@ static FusedPlan* fused_plan(int dev, int sm_count) {
     p.ready = true;
     int coop = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return &p;
-    if (cudaFuncSetAttribute(k_gk_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBudget) !=
-        cudaSuccess) {
-        cudaGetLastError();
-        return &p;
-    }
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused, kFusedThreads, kFusedSmemBudget) !=
-            cudaSuccess || occ < 1) {
-        cudaGetLastError();
-        return &p;
-    }
+    if (!fused_kernel_ready<true>() || !fused_kernel_ready<false>()) return &p;
     p.grid = sm_count < kFusedMaxGrid ? sm_count : kFusedMaxGrid;
     p.usable = true;
     return &p;
@@ -705,24 +954,42 @@ static FusedGeometry fused_geometry(int64_t d, int grid) {
     return q;
 }
 
+// Whether the call counts during phase A against predicted thresholds: on vectors large enough
+// for the prediction to arrive early in a CTA's run (a test hook can force either answer).
+static int wants_prediction(const FusedGeometry& geo, int64_t d) {
+    const bool possible = (d >> 7) >= 1;   // one block of 32 float4 at least
+    const int knob = host_knob(kKnobPrediction);
+    if (knob == 0 || !possible) return 0;
+    if (knob == 1) return 1;
+    return (int64_t)geo.n_rows >= (int64_t)kPredMinRows * geo.G ? 1 : 0;
+}
+
 // The one place that builds the kernel's argument list (types checked by the compiler).
-static cudaError_t launch_fused(const FusedGeometry& geo, cudaStream_t st, const float* g, float* eps, int64_t d,
-                                int64_t k, double z, Ctrl* ctrl, double2* partials, unsigned int* cta_counts,
+// eps == nullptr launches the operator form.
+static cudaError_t launch_fused(const FusedGeometry& geo, cudaStream_t st, const float* src, float* eps, int64_t d,
+                                int64_t k, double z, Ctrl* ctrl, double2* partials, double2* spart,
                                 unsigned int* bars, unsigned int* rowcnt, int32_t* idx_out, float* val_out,
                                 int64_t* nnz_out, int64_t cap, unsigned long long* trace) {
     int n_rows = geo.n_rows, u_slots = geo.u_slots, table_rows = geo.table_rows;
-    void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&n_rows, (void*)&u_slots,
-                    (void*)&table_rows, (void*)&ctrl, (void*)&partials, (void*)&cta_counts, (void*)&bars,
-                    (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap, (void*)&trace};
-    static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused takes 18 arguments");
-    return cudaLaunchCooperativeKernel((const void*)k_gk_fused, dim3((unsigned)geo.G), dim3(kFusedThreads), args,
+    int predict = wants_prediction(geo, d);
+    unsigned int bar_target = (unsigned int)geo.G + (unsigned int)host_knob(kKnobExtraArrivals);
+    void* args[] = {(void*)&src, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&n_rows, (void*)&u_slots,
+                    (void*)&table_rows, (void*)&predict, (void*)&bar_target, (void*)&ctrl, (void*)&partials,
+                    (void*)&spart, (void*)&bars, (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out,
+                    (void*)&cap, (void*)&trace};
+    static_assert(sizeof(args) / sizeof(args[0]) == 20, "k_gk_fused takes 20 arguments");
+    // the two instances have the same parameter list; naming them keeps the types checked
+    void (*kern)(const float*, float*, int64_t, int64_t, double, int, int, int, int, unsigned int, Ctrl*, double2*,
+                 double2*, unsigned int*, unsigned int*, int32_t*, float*, int64_t*, int64_t, unsigned long long*) =
+        eps != nullptr ? k_gk_fused<true> : k_gk_fused<false>;
+    return cudaLaunchCooperativeKernel((const void*)kern, dim3((unsigned)geo.G), dim3(kFusedThreads), args,
                                        geo.smem, st);
 }
 
 // Returns GK_OK when the fused kernel was enqueued, 1 when it cannot be used on
 // this device or for this call (the caller then takes the three-kernel path),
 // or an error.
-int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                      float* val_out, int64_t* nnz_out, cudaStream_t st) {
     int dev = 0;
     GK_CUDA_TRY(cudaGetDevice(&dev));
@@ -734,8 +1001,9 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
     const double z = normal_quantile_upper(1.0 - pq);
     ws->last_grid = (int)geo.G;
     stage_mark(ws, st, 0);
-    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ws->ctrl, ws->partials, ws->cta_counts, ws->bars, ws->rowcnt,
-                             idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
+    // the sample sums sit behind the per-CTA partials (at most kFusedGridCap of them)
+    GK_CUDA_TRY(launch_fused(geo, st, src, eps, d, k, z, ws->ctrl, ws->partials, ws->partials + kFusedGridCap, ws->bars,
+                             ws->rowcnt, idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_fused = true;
@@ -753,8 +1021,8 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
 // service that forbids device allocations after start-up because cudaMalloc
 // synchronises the whole device, or a step that has to behave the same on its
 // first and on its millionth call.  For them the scratch of the fused kernel
-// (control block, per-CTA partial sums, per-CTA candidate counts, barrier
-// counters, one word per row of the vector) lives in the fixed array below
+// (control block, per-CTA partial sums, barrier counters and global counts,
+// one word per row of the vector) lives in the fixed array below
 // instead of a workspace obtained from cudaMalloc.  The array is part of the
 // library image: every GPU that loads the library holds these 544 KB until the
 // process exits.
@@ -762,13 +1030,12 @@ int enqueue_gk_fused(Workspace* ws, const float* g, float* eps, int64_t d, int64
 namespace gk {
 
 constexpr size_t kStaticCtrlBytes = (sizeof(Ctrl) + 255) / 256 * 256;
-constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap;                // 8 KB
-constexpr size_t kStaticCountBytes = sizeof(unsigned int) * kFusedGridCap * kNumCand;  // 20 KB
-constexpr size_t kStaticBarBytes = 256;
+constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap * 3;   // 24 KB: partial sums, then sample sums
+constexpr size_t kStaticBarBytes = sizeof(unsigned int) * kBarWords;          // 256 bytes
 constexpr size_t kStaticHeadBytes = 32 * 1024;             // everything but the per-row words
 constexpr int kStaticRowCap = 1 << 17;                     // rows of 4096 elements: d up to 2^29
 constexpr size_t kStaticScratchBytes = kStaticHeadBytes + sizeof(unsigned int) * kStaticRowCap;  // 544 KB
-static_assert(kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes + kStaticBarBytes <= kStaticHeadBytes,
+static_assert(kStaticCtrlBytes + kStaticPartialBytes + kStaticBarBytes <= kStaticHeadBytes,
               "static scratch too small");
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -816,23 +1083,21 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
 
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(ss->base);
     double2* partials = reinterpret_cast<double2*>(ss->base + kStaticCtrlBytes);
-    unsigned int* cta_counts = reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes);
-    unsigned int* bars =
-        reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes + kStaticCountBytes);
+    unsigned int* bars = reinterpret_cast<unsigned int*>(ss->base + kStaticCtrlBytes + kStaticPartialBytes);
 
     unsigned int* rowcnt = reinterpret_cast<unsigned int*>(ss->base + kStaticHeadBytes);
 
     const FusedGeometry geo = fused_geometry(d, plan->grid);
     // more CTAs or rows than the fixed array has slots for, or more rows per CTA than the kernel takes
     if (geo.G > kFusedGridCap || geo.n_rows > kStaticRowCap || !geo.fits) return GK_ERR_LIMIT;
-    // The array keeps what the last call left.  The barrier counters must start at zero; the
-    // kernel resets them when it ends, but a call that was cut short would not have.
+    // The array keeps what the last call left.  The barrier counters and the global counts must
+    // start at zero; the kernel resets them when it ends, but a call that was cut short would not have.
     GK_CUDA_TRY(cudaMemsetAsync(bars, 0, kStaticBarBytes, st));
     const double pq = 1.0 - (double)k / (double)d;
     const double z = normal_quantile_upper(1.0 - pq);
     unsigned long long* trace = nullptr;  // no trace array in the fixed scratch
-    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, cta_counts, bars, rowcnt, idx_out, val_out,
-                             nnz_out, output_capacity(d), trace));
+    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, partials + kFusedGridCap, bars, rowcnt, idx_out,
+                             val_out, nnz_out, output_capacity(d), trace));
     note_launch();
     return GK_OK;
 }

@@ -59,7 +59,7 @@ static Layout layout_for(int64_t d, int32_t S) {
     L.partials = at;    at = align_up(at + sizeof(double2) * kMaxPartials, 256);
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
     L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
-    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 16, 256);
+    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 64, 256);
     L.cta_trace = at;   at = align_up(at + sizeof(unsigned long long) * kFusedGridCap * 8, 256);
     L.rowcnt = at;      at = align_up(at + sizeof(unsigned int) * 2 * ((size_t)(d >> 12) + 2), 256);
     L.tile_status = at; at = align_up(at + sizeof(unsigned long long) * (size_t)num_compact_tiles(d), 256);
@@ -129,6 +129,31 @@ static std::map<int, HostStage> g_stage;
 static std::atomic<int> g_path{0};
 int selected_path() { return g_path.load(std::memory_order_relaxed); }
 
+// Test hooks: setters registered by the translation units that hold device-side knobs, and
+// the host-side knobs themselves.
+struct KnobRegistry {
+    std::mutex mu;
+    KnobSetter fn[32];
+    int n = 0;
+};
+static KnobRegistry& knob_registry() {
+    static KnobRegistry r;   // constructed on first use: units register during static initialisation
+    return r;
+}
+int register_knob_setter(KnobSetter fn) {
+    KnobRegistry& r = knob_registry();
+    std::lock_guard<std::mutex> lock(r.mu);
+    if (r.n < 32) r.fn[r.n++] = fn;
+    return r.n;
+}
+static std::atomic<int> g_host_knob[kKnobCount] = {};
+static std::atomic<bool> g_host_knob_set[kKnobCount] = {};
+int host_knob(int key) {
+    if (key < 0 || key >= kKnobCount) return 0;
+    if (!g_host_knob_set[key].load()) return key == kKnobPrediction ? -1 : 0;
+    return g_host_knob[key].load();
+}
+
 }  // namespace gk
 
 using namespace gk;
@@ -142,6 +167,19 @@ extern "C" int gk_set_capacity(int64_t cap) {
 extern "C" int gk_set_path(int path) {
     if (path < 0 || path > 1) return GK_ERR_SIZE;
     g_path.store(path);
+    return GK_OK;
+}
+
+extern "C" int gk_debug_set(int key, int64_t value) {
+    if (key < 0 || key >= kKnobCount || value < -1 || value > 2147483647ll) return GK_ERR_SIZE;
+    g_host_knob[key].store((int)value);
+    g_host_knob_set[key].store(true);
+    KnobRegistry& r = knob_registry();
+    std::lock_guard<std::mutex> lock(r.mu);
+    for (int i = 0; i < r.n; ++i) {
+        const int e = r.fn[i](key, (int)value);
+        if (e != 0) return cuda_fail((cudaError_t)e);
+    }
     return GK_OK;
 }
 
@@ -190,6 +228,18 @@ extern "C" int gk_last_segment_stats(gk_stream_t stream, int32_t S, gk_stats* ho
         host_out[s].status |= total.status;
         if (!(total.status & (GK_DEV_TRUNCATED | GK_DEV_TIMEOUT))) host_out[s].emitted = host_out[s].nnz;
     }
+    return GK_OK;
+}
+
+extern "C" int gk_last_path_info(gk_stream_t stream, int64_t* host_out) {
+    if (!host_out) return GK_ERR_NULL;
+    Workspace* ws = find_workspace((cudaStream_t)stream);
+    if (!ws) return GK_ERR_NULL;
+    GK_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    unsigned int v[4];
+    GK_CUDA_TRY(cudaMemcpy(v, ws->ctrl->path_info, sizeof(v), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 4; ++i) host_out[i] = (int64_t)v[i];
+    host_out[4] = ws->last_fused ? ws->last_grid : 0;
     return GK_OK;
 }
 

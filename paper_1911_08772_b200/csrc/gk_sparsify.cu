@@ -30,8 +30,10 @@ __device__ __forceinline__ Alg1State state_of(Ctrl* ctrl) {
 }
 
 // ---------------------------------------------------------------------------
-// Kernel A.  Grid-stride over float4; every CTA writes one partial.
+// Kernel A.  Grid-stride over float4; every CTA writes one partial.  ACC: u = g + eps is
+// formed and stored over eps; !ACC: g is the vector u itself and nothing is stored.
 // ---------------------------------------------------------------------------
+template <bool ACC>
 __global__ void __launch_bounds__(kAccThreads)
 k_accumulate_stats(const float* __restrict__ g, float* __restrict__ eps, int64_t d, int64_t k, double z,
                    Ctrl* __restrict__ ctrl, double2* __restrict__ partials,
@@ -56,16 +58,21 @@ k_accumulate_stats(const float* __restrict__ g, float* __restrict__ eps, int64_t
 #pragma unroll
         for (int j = 0; j < kAccUnroll; ++j) {
             const int64_t ii = i + j * gstride;
-            if (ii < n4) { a[j] = ld_stream(g4 + ii); b[j] = ld_stream(e4 + ii); }
+            if (ii < n4) {
+                a[j] = ld_stream(g4 + ii);
+                b[j] = ACC ? ld_stream(e4 + ii) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
 #pragma unroll
         for (int j = 0; j < kAccUnroll; ++j) {
             const int64_t ii = i + j * gstride;
             if (ii < n4) {
-                float4 u;
-                u.x = a[j].x + b[j].x; u.y = a[j].y + b[j].y;
-                u.z = a[j].z + b[j].z; u.w = a[j].w + b[j].w;
-                e4[ii] = u;
+                float4 u = a[j];
+                if (ACC) {
+                    u.x = a[j].x + b[j].x; u.y = a[j].y + b[j].y;
+                    u.z = a[j].z + b[j].z; u.w = a[j].w + b[j].w;
+                    e4[ii] = u;
+                }
                 const double x0 = (double)u.x - c, x1 = (double)u.y - c;
                 const double x2 = (double)u.z - c, x3 = (double)u.w - c;
                 s0 += x0; q0 = fma(x0, x0, q0);
@@ -78,8 +85,8 @@ k_accumulate_stats(const float* __restrict__ g, float* __restrict__ eps, int64_t
     // ragged tail (d not a multiple of 4)
     if (blockIdx.x == 0 && tid < (int)(d & 3)) {
         const int64_t i = (n4 << 2) + tid;
-        const float u = g[i] + eps[i];
-        eps[i] = u;
+        const float u = ACC ? g[i] + eps[i] : g[i];
+        if (ACC) eps[i] = u;
         const double x = (double)u - c;
         s0 += x; q0 = fma(x, x, q0);
     }
@@ -199,8 +206,9 @@ static int reduction_grid(const Workspace* ws, int64_t d, int threads, int unrol
     return (int)(want < cap ? want : cap);
 }
 
-// Enqueue the three-kernel (look-back) path on an already validated call.
-int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
+// Enqueue the three-kernel (look-back) path on an already validated call.  eps == nullptr:
+// the operator form (src = u, read only).
+int enqueue_gk_three_kernel(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k,
                         int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st) {
     const int n_tiles = (int)num_compact_tiles(d);
     double z = -INFINITY;
@@ -210,19 +218,29 @@ int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d
     }
     const int grid_a = reduction_grid(ws, d, kAccThreads, kAccUnroll, 4);
     stage_mark(ws, st, 0);
-    k_accumulate_stats<<<grid_a, kAccThreads, 0, st>>>(g, eps, d, k, z, ws->ctrl, ws->partials,
-                                                       ws->tile_status, n_tiles);
+    if (eps != nullptr)
+        k_accumulate_stats<true><<<grid_a, kAccThreads, 0, st>>>(src, eps, d, k, z, ws->ctrl, ws->partials,
+                                                                 ws->tile_status, n_tiles);
+    else
+        k_accumulate_stats<false><<<grid_a, kAccThreads, 0, st>>>(src, nullptr, d, k, z, ws->ctrl, ws->partials,
+                                                                  ws->tile_status, n_tiles);
     note_launch();
     stage_mark(ws, st, 1);
+    float* uvec = eps != nullptr ? eps : const_cast<float*>(src);   // the operator form never writes it
     if (k < d) {
         const int grid_b = reduction_grid(ws, d, kCntThreads, kCntUnroll, 4);
-        k_count_candidates<<<grid_b, kCntThreads, 0, st>>>(eps, d, k, ws->ctrl);
+        k_count_candidates<<<grid_b, kCntThreads, 0, st>>>(uvec, d, k, ws->ctrl);
         note_launch();
     }
     stage_mark(ws, st, 2);
-    GK_CUDA_TRY(launch_compaction(k_compact_threshold<false>, n_tiles, ws->sm_count, st, eps, d, ws->ctrl,
-                                  ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
-                                  (const int64_t*)nullptr, 0, (const float*)nullptr));
+    if (eps != nullptr)
+        GK_CUDA_TRY(launch_compaction(k_compact_threshold<false, true>, n_tiles, ws->sm_count, st, uvec, d, ws->ctrl,
+                                      ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
+                                      (const int64_t*)nullptr, 0, (const float*)nullptr));
+    else
+        GK_CUDA_TRY(launch_compaction(k_compact_threshold<false, false>, n_tiles, ws->sm_count, st, uvec, d, ws->ctrl,
+                                      ws->tile_status, n_tiles, idx_out, val_out, nnz_out, output_capacity(d),
+                                      (const int64_t*)nullptr, 0, (const float*)nullptr));
     note_launch();
     stage_mark(ws, st, 3);
     ws->last_fused = false;
@@ -233,13 +251,14 @@ int enqueue_gk_three_kernel(Workspace* ws, const float* g, float* eps, int64_t d
 
 // Enqueue one step by the selected path: the fused cooperative kernel unless it
 // cannot be used on this device (or for this call), else the three-kernel path.
-int enqueue_gk_sparsify(Workspace* ws, const float* g, float* eps, int64_t d, int64_t k,
+// eps == nullptr: the operator form on src = u.
+int enqueue_gk_sparsify(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k,
                         int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st) {
     if (selected_path() != 1) {
-        const int rc = enqueue_gk_fused(ws, g, eps, d, k, idx_out, val_out, nnz_out, st);
+        const int rc = enqueue_gk_fused(ws, src, eps, d, k, idx_out, val_out, nnz_out, st);
         if (rc != 1) return rc;
     }
-    return enqueue_gk_three_kernel(ws, g, eps, d, k, idx_out, val_out, nnz_out, st);
+    return enqueue_gk_three_kernel(ws, src, eps, d, k, idx_out, val_out, nnz_out, st);
 }
 
 }  // namespace gk
@@ -252,4 +271,16 @@ extern "C" int gk_sparsify(const float* g, float* eps, int64_t d, int64_t k, int
     const int wrc = gk::acquire_workspace(d, 1, (cudaStream_t)stream, &ws);
     if (wrc != GK_OK) return wrc;
     return gk::enqueue_gk_sparsify(ws, g, eps, d, k, idx_out, val_out, nnz_out, (cudaStream_t)stream);
+}
+
+extern "C" int gk_select(const float* u, int64_t d, int64_t k, int32_t* idx_out, float* val_out,
+                         int64_t* nnz_out, gk_stream_t stream) {
+    if (!u || !idx_out || !val_out || !nnz_out) return GK_ERR_NULL;
+    if (d < 1 || d > 2147483647ll) return GK_ERR_SIZE;
+    if (k < 1 || k > d) return GK_ERR_K;
+    if ((uintptr_t)u & 15u) return GK_ERR_ALIGN;
+    gk::Workspace* ws = nullptr;
+    const int wrc = gk::acquire_workspace(d, 1, (cudaStream_t)stream, &ws);
+    if (wrc != GK_OK) return wrc;
+    return gk::enqueue_gk_sparsify(ws, u, nullptr, d, k, idx_out, val_out, nnz_out, (cudaStream_t)stream);
 }

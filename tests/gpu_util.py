@@ -121,6 +121,23 @@ def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, c
     return eps_new, st
 
 
+def check_gk_select(step: DeviceStep, u: np.ndarray, k: int, check_counts=True):
+    """gk_select on the device against the oracle: Algorithm 1 on u as given, u untouched."""
+    step.g.copy_(torch.from_numpy(u))
+    step.arm()
+    gk.gk_select(step.g, k, step.idx[:step.cap], step.val[:step.cap], step.nnz[:1])
+    idx, val, n = step.outputs()
+    st = gk.gk_last_stats()
+    assert np.array_equal(bits(step.g.cpu().numpy()), bits(u)), "u modified"
+    # the operator is the sparsifier's selection with a neutral residual coming in; the residual
+    # the oracle would leave is u with the selected entries cleared
+    zero = np.full_like(u, -0.0)    # x + (-0) == x for every x, -0 included: the oracle sees u itself
+    u_cleared = u.copy()
+    u_cleared[idx] = 0.0
+    compare_with_oracle(u, zero, k, idx, val, n, st, u_cleared, step.cap, check_counts)
+    return st
+
+
 def check_segmented_step(step: DeviceStep, g, eps_in, offsets, seg_k, dev_off, dev_k, dev_seg_nnz):
     d = g.shape[0]
     S = offsets.shape[0] - 1

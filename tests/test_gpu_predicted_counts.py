@@ -1,0 +1,157 @@
+"""The fused kernel's counting against predicted thresholds (Algorithm 1's counts taken while
+the vector streams in): whatever the prediction does -- holds, misses, is refused, or the
+rounds leave the six upper candidates -- the statistics, the per-round counts, the pairs and
+the residual must equal the oracle's.  gk_debug_set(4, 1) switches the prediction on for
+vectors far smaller than the size from which the library uses it by itself."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1911_08772_b200 import binding as gk
+from paper_1911_08772_b200 import workloads as wl
+
+from gpu_util import DeviceStep, bits, check_gk_step
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    from paper_1911_08772_b200 import build
+    build.build()
+    gk.load()
+    gk.gk_set_capacity(0)
+    gk.gk_set_path(0)
+    yield
+    gk.gk_debug_set(gk.KNOB_PREDICTION, -1)
+
+
+@pytest.fixture
+def predicted():
+    gk.gk_debug_set(gk.KNOB_PREDICTION, 1)
+    yield
+    gk.gk_debug_set(gk.KNOB_PREDICTION, -1)
+
+
+def _rows_per_cta(d):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    return (d // 4096) // sms
+
+
+@pytest.mark.parametrize("d", [2_000_003, 8_000_003, 20_000_001])
+@pytest.mark.parametrize("dist", ["normal", "laplace", "segments"])
+def test_prediction_holds_on_bell_shaped_vectors(d, dist, predicted):
+    k = wl.ceil_k(d, 1, 1000)
+    part = wl.seeded_partition(d, 23) if dist == "segments" else None
+    step = DeviceStep(d)
+    eps = np.zeros(d, dtype=np.float32)
+    used = 0
+    for t in range(3):
+        g = {"normal": lambda: wl.normal(d, 1e-3, step=90 + t),
+             "laplace": lambda: wl.laplace(d, 1e-3, step=90 + t),
+             "segments": lambda: wl.segmented_normal(part, step=90 + t)}[dist]()
+        eps, st = check_gk_step(step, g, eps, k)
+        with_pred, held, recount, left, ctas = gk.gk_last_path_info()
+        assert ctas > 0 and recount == 0
+        used += held
+        if _rows_per_cta(d) >= 6:
+            # the sample totals arrive within the first rows of every CTA, and on data like these
+            # the bands hold everywhere
+            assert with_pred == ctas and held == ctas, (with_pred, held, ctas)
+    assert used > 0 or _rows_per_cta(d) < 6
+
+
+@pytest.mark.parametrize("rho", ["1e-4", "1e-2"])
+def test_prediction_at_other_densities(rho, predicted):
+    d = 12_000_017
+    k = wl.ceil_k(d, *wl.RHO[rho])
+    step = DeviceStep(d)
+    eps = np.zeros(d, dtype=np.float32)
+    for t in range(2):
+        eps, st = check_gk_step(step, wl.normal(d, 1.0, step=95 + t), eps, k)
+    assert gk.gk_last_path_info()[1] > 0
+
+
+def test_rounds_that_leave_the_upper_candidates_are_counted_again_in_full(predicted):
+    # uniform values: sigma = a / sqrt 3, the first threshold lies beyond every magnitude, the
+    # first count is 0 and the rounds go down to thres0 / 2 and below
+    d = 9_000_011
+    rng = wl.misc_rng(31)
+    g = rng.uniform(-1.0, 1.0, size=d).astype(np.float32)
+    step = DeviceStep(d)
+    _, st = check_gk_step(step, g, np.zeros(d, np.float32), wl.ceil_k(d, 1, 1000))
+    with_pred, held, recount, left, ctas = gk.gk_last_path_info()
+    assert held > 0 and recount == 1
+    assert st.counts[0] == 0 and st.rounds == 4
+
+
+def test_a_sample_that_misleads_is_found_out(predicted):
+    # the blocks of 128 elements the kernel samples are spread evenly; a vector whose even 4096-element
+    # rows are quiet and whose odd ones are loud in a pattern the even sample cannot see: the
+    # prediction may hold or miss, the result must not care.  Here half of the vector is ten
+    # times wider than the other half, in alternating stretches of 1000 elements.
+    d = 8_500_003
+    g = wl.normal(d, 1e-3, step=97)
+    scale = np.where((np.arange(d) // 1000) % 2 == 0, np.float32(1.0), np.float32(10.0))
+    g = (g * scale).astype(np.float32)
+    step = DeviceStep(d)
+    check_gk_step(step, g, np.zeros(d, np.float32), wl.ceil_k(d, 1, 1000))
+    # and a vector whose sampled blocks are all zero: the sample's variance is zero and the
+    # prediction is refused
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n4 = d >> 2
+    nblk = n4 >> 5
+    j = np.arange(sms * 32, dtype=np.int64)
+    blk = (j * nblk) // (sms * 32)
+    g2 = wl.normal(d, 1e-3, step=98)
+    for b in blk:
+        g2[b * 128:(b + 1) * 128] = 0.0
+    check_gk_step(step, g2, np.zeros(d, np.float32), wl.ceil_k(d, 1, 1000))
+    assert gk.gk_last_path_info()[0] == 0
+    # the same blocks at ten times the vector's scale: the sample overstates sigma, the bands miss
+    g3 = wl.normal(d, 1e-3, step=99)
+    for b in blk:
+        g3[b * 128:(b + 1) * 128] *= np.float32(1.5)
+    check_gk_step(step, g3, np.zeros(d, np.float32), wl.ceil_k(d, 1, 1000))
+    with_pred, held, recount, left, ctas = gk.gk_last_path_info()
+    assert with_pred > 0 and held == 0
+
+
+def test_heavy_tails_and_outliers(predicted):
+    d = 10_000_019
+    step = DeviceStep(d)
+    eps = np.zeros(d, dtype=np.float32)
+    for t in range(2):
+        eps, st = check_gk_step(step, wl.student_t3_outliers(d, step=80 + t), eps, wl.ceil_k(d, 1, 1000))
+    eps = np.zeros(d, dtype=np.float32)
+    for t in range(2):
+        eps, st = check_gk_step(step, wl.laplace_mixture(d, step=82 + t), eps, wl.ceil_k(d, 1, 1000))
+
+
+def test_negative_and_shifted_thresholds(predicted):
+    d = 7_000_001
+    g = wl.normal(d, 1e-3, step=85)
+    z = np.zeros(d, np.float32)
+    step = DeviceStep(d)
+    _, st = check_gk_step(step, (g - np.float32(5.0)).astype(np.float32), z, 7000)     # thres0 < 0
+    assert st.nnz == d and gk.gk_last_path_info()[0] == 0
+    check_gk_step(step, (g + np.float32(0.5)).astype(np.float32), z, 7000)             # one-sided tail: stops at once
+    check_gk_step(step, np.zeros(d, np.float32), z, 7000)                              # sigma = 0
+
+
+def test_with_and_without_prediction_give_the_same_bits():
+    d = 11_000_003
+    k = wl.ceil_k(d, 1, 1000)
+    g = wl.laplace_mixture(d, step=86)
+    e = wl.normal(d, 1e-3, step=87)
+    outs = []
+    try:
+        for mode in (0, 1, 1, 0):
+            gk.gk_debug_set(gk.KNOB_PREDICTION, mode)
+            step = DeviceStep(d)
+            eps_new, st = check_gk_step(step, g, e, k)
+            outs.append((bits(eps_new).copy(), st))
+    finally:
+        gk.gk_debug_set(gk.KNOB_PREDICTION, -1)
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0]) and o[1] == outs[0][1]
