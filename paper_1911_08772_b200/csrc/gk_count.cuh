@@ -15,37 +15,30 @@ __device__ __forceinline__ float gt_as_float(float a, float c) {
 
 // Candidates LO..HI-1 (in ascending order of value) against the four magnitudes of one
 // float4.  The counters are floats: exact up to 2^24 per thread, far above a thread's share.
-template <int LO, int HI>
+template <int LO, int HI, int N>
 __device__ __forceinline__ void count_tier(const float a0, const float a1, const float a2, const float a3,
-                                           const float (&cs)[kNumCand], float (&acc)[kNumCand]) {
+                                           const float (&cs)[N], float (&acc)[N]) {
 #pragma unroll
     for (int j = LO; j < HI; ++j)
         acc[j] += (gt_as_float(a0, cs[j]) + gt_as_float(a1, cs[j])) + (gt_as_float(a2, cs[j]) + gt_as_float(a3, cs[j]));
 }
 
-// rm: the segment's largest magnitude (top 16 bits, rounded up).  A candidate whose top 16
-// bits (rounded down) are not below rm cannot be exceeded by any element of the segment, nor
+// rm: the cell's largest magnitude (top 16 bits, rounded up).  A candidate whose top 16
+// bits (rounded down) are not below rm cannot be exceeded by any element of the cell, nor
 // can any larger candidate: candidates 0..1, 2..4, 5..6 and 7..9 (in ascending order) are
-// evaluated only as far as the segment's maximum reaches.
+// evaluated only as far as the cell's maximum reaches.
 struct Tiers { unsigned int t0, t2, t5, t7; };
-// FIRST = 0: all ten candidates.  FIRST = 4: only candidates 4..9 (the caller then sets tier.t0
-// to the limit of candidate 4): the counters of candidates 0..3 are not touched.
-template <int FIRST = 0>
 __device__ __forceinline__ void count_float4(const float4 v, const unsigned int rm, const float (&cs)[kNumCand],
                                              const Tiers& tier, float (&acc)[kNumCand]) {
-    static_assert(FIRST == 0 || FIRST == 4, "the tiers start at candidate 0 or 4");
     if (rm <= tier.t0) return;  // warp-uniform, as are the tests below
     const float a0 = fabsf(v.x), a1 = fabsf(v.y), a2 = fabsf(v.z), a3 = fabsf(v.w);
-    if (FIRST == 0) {
-        count_tier<0, 2>(a0, a1, a2, a3, cs, acc);
-        if (rm <= tier.t2) return;
+    count_tier<0, 2>(a0, a1, a2, a3, cs, acc);
+    if (rm > tier.t2) {
         count_tier<2, 5>(a0, a1, a2, a3, cs, acc);
-    } else {
-        count_tier<4, 5>(a0, a1, a2, a3, cs, acc);
-    }
-    if (rm > tier.t5) {
-        count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
-        if (rm > tier.t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
+        if (rm > tier.t5) {
+            count_tier<5, 7>(a0, a1, a2, a3, cs, acc);
+            if (rm > tier.t7) count_tier<7, kNumCand>(a0, a1, a2, a3, cs, acc);
+        }
     }
 }
 

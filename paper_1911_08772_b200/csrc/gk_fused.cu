@@ -56,7 +56,9 @@
 // launched cooperatively, so all CTAs are resident and the waits do end.
 #include <math.h>
 
+#include <cstddef>
 #include <mutex>
+#include <type_traits>
 
 #include "gk_alg1.cuh"
 #include "gk_common.cuh"
@@ -79,8 +81,14 @@ constexpr int kStageCap = kRing * kRowF4 * 4;
 
 // Counting during phase A (prediction of the thresholds from a sample).
 constexpr int kUpper = 6;               // candidates thres0 * {3/4, 1, 9/8, 3/2, 9/4, 27/8}: sorted places 4..9
-constexpr int kPredMinRows = 10;        // rows per CTA from which on the prediction is tried
-constexpr int kPredPollFirst = 2;       // first row before which a CTA looks for the sample totals
+// Rows per CTA from which on the prediction is tried without being asked for (39 M elements on 148
+// SMs).  Measured on B200: at 110 rows per CTA (2^26 elements) the streaming phase is bound by HBM and
+// takes the extra work for free (200 -> 177 us per call); at 42 rows (25.6 M elements, half of eps
+// served by L2) it has no issue slots to spare and the two ways take the same time; below, the
+// prediction costs more than it saves.
+constexpr int kPredMinRows = 64;
+constexpr int kPredMaxRows = 511;       // ... and up to which: a thread's counts (4 per row) are kept in 13 bits
+constexpr float kPackScale = 8192.f;    // two counts in one float: lo + 8192 * hi, exact below 2^24
 constexpr int kSampleElems = kFusedThreads * 4;   // sample elements per CTA: one float4 per thread
 constexpr double kPredSigmas = 3.5;     // half width of the bands in standard errors of the predicted threshold
 constexpr double kPredSlack = 5e-4;     // added to the relative half width
@@ -100,11 +108,11 @@ constexpr int kBarStats = 0;      // barrier after phase A
 constexpr int kBarCounts = 1;     // barrier after phase B
 constexpr int kBarExit = 2;       // CTAs that have left
 constexpr int kBarRows = 3;       // barrier inside phase C
-constexpr int kBarPublished = 9;  // CTAs whose sample sums are in place
 constexpr int kBarInvalid = 14;   // candidates (bit = index) that some CTA has not counted
 constexpr int kBarCounts2 = 15;   // barrier after the second, full count
 constexpr int kBarTotals = 16;    // 2 x kNumCand words: the global counts of the first and the second count
 constexpr int kBarInfo = 36;      // 4 words: what Ctrl::path_info reports, collected during the call
+constexpr int kBarSample = 48;    // 4 doubles: the sample's power sums over all CTAs; then a word: CTAs that are in
 constexpr int kBarWords = 64;
 
 struct __align__(128) FusedShared {
@@ -118,20 +126,27 @@ struct __align__(128) FusedShared {
     float thr_sel;
     int chosen;
     int ok;
-    int poll[2];                        // the sample totals were complete when row r (parity) began
-    int pred_ok;                        // a usable prediction was formed
+    unsigned int samp_n;                // warps whose sums are in
+    int pred_ready;                     // 0: no word yet; 1: the predicted bands stand; 2: no prediction
     int fast;                           // this CTA's bands hold the exact candidates
     int recount;                        // the rounds need a candidate that some CTA has not counted
     gk_stats stats;
     unsigned int wsum[kFusedWarps];
-    unsigned int roundtot[kTableMaxRows];  // survivors in each round of rows (G consecutive rows)
+    // survivors in each round of rows (G consecutive rows); before phase C the first 1 KB holds
+    // the warps' sample sums as double2, hence the alignment
+    alignas(16) unsigned int roundtot[kTableMaxRows];
     unsigned int rowpre[kTableMaxRows];    // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
     unsigned int n_staged;                 // survivors put aside in phase C
 };
 
-static_assert((sizeof(FusedShared) + 1023) / 1024 * 1024 + kFusedSmemBudget <= 232448,
-              "over the 227 KB of shared memory per CTA (the dynamic part starts on a 1 KB boundary)");
+static_assert(offsetof(FusedShared, roundtot) % 16 == 0 && sizeof(unsigned int) * kTableMaxRows >= 64 * kFusedWarps,
+              "the sample slots (two double2 per warp) borrow roundtot");
+// FusedShared sits at the front of the dynamic shared memory, the rows behind it on a 1 KB boundary
+constexpr int kFusedStaticBytes = 11264;
+static_assert(sizeof(FusedShared) <= kFusedStaticBytes && kFusedStaticBytes % 1024 == 0 &&
+                  kFusedStaticBytes + kFusedSmemBudget <= 232448,
+              "over the 227 KB of shared memory per CTA");
 
 __device__ __forceinline__ unsigned int mask_above(const float4 v, const float thr) {
     return (unsigned)(fabsf(v.x) > thr) | ((unsigned)(fabsf(v.y) > thr) << 1) |
@@ -148,467 +163,343 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
 // (n sample elements).  The half width is kPredSigmas standard errors of mu + sigma z, with the
 // standard error of sigma taken from the sample's own fourth moment (heavy tails widen the
 // bands by themselves), plus a small slack.  Returns false when no useful prediction exists.
-__device__ inline bool predict_bands(double s1, double s2, double s3, double s4, double n, double pv, double z,
+__device__ __noinline__ bool predict_bands(double s1, double s2, double s3, double s4, double n, double pv, double z,
                                      float* plo, float* phi) {
-    const double m1 = s1 / n, r2 = s2 / n, r3 = s3 / n, r4 = s4 / n;
+    const double inv_n = 1.0 / n;
+    const double m1 = s1 * inv_n, r2 = s2 * inv_n, r3 = s3 * inv_n, r4 = s4 * inv_n;
     const double var_p = r2 - m1 * m1;                    // population variance of the sample
     if (!(var_p > 0.0) || !(n > 2.0)) return false;
-    const double var = var_p * n / (n - 1.0);
     const double c4 = r4 - 4.0 * m1 * r3 + 6.0 * m1 * m1 * r2 - 3.0 * m1 * m1 * m1 * m1;   // central fourth moment
-    const double kurt = c4 / (var_p * var_p);
-    const double sigma = sqrt(var);
-    const double th = (pv + m1) + sigma * z;
+    // from here on single precision is plenty: the half width is a bound, not a result
+    const float nf = (float)n, zf = (float)z;
+    const float var = (float)var_p * (nf / (nf - 1.0f));
+    const float kurt = (float)c4 / ((float)var_p * (float)var_p);
+    const float sigma = sqrtf(var);
+    const double th = (pv + m1) + (double)sigma * z;
     if (!(th > 0.0) || !(th < 3.0e38)) return false;
-    const double se_sigma = 0.5 * sqrt(fmax(kurt - 1.0, 0.0) / n) * sigma;   // standard error of sigma
-    const double se_th = sqrt(var / n + z * z * se_sigma * se_sigma);
-    const double delta = kPredSigmas * se_th / th + kPredSlack;
-    if (!(delta < kPredMaxDelta)) return false;
+    const float se_sigma = 0.5f * sqrtf(fmaxf(kurt - 1.0f, 0.0f) / nf) * sigma;   // standard error of sigma
+    const float se_th = sqrtf(var / nf + zf * zf * se_sigma * se_sigma);
+    const float delta = (float)kPredSigmas * se_th / (float)th + (float)kPredSlack;
+    if (!(delta < (float)kPredMaxDelta)) return false;
     const double f[kUpper] = {0.75, 1.0, 1.125, 1.5, 2.25, 3.375};
+    const double dn = 1.0 - (double)delta, up = 1.0 + (double)delta;
 #pragma unroll
     for (int j = 0; j < kUpper; ++j) {
-        plo[j] = __double2float_rd(th * f[j] * (1.0 - delta));
-        phi[j] = __double2float_ru(th * f[j] * (1.0 + delta));
+        plo[j] = __double2float_rd(th * f[j] * dn);
+        phi[j] = __double2float_ru(th * f[j] * up);
     }
     return phi[kUpper - 1] < 3.0e38f;
 }
 
-// ACC: the sparsifier (src = g, u = g + eps is formed, stored over eps and cleared where
-// selected); !ACC: the operator on a given vector (src = u, read only; eps is not used).
-// n_rows: rows of 1024 float4 in the whole vector; CTA c owns rows c, c + G, c + 2G, ...
-// (G = gridDim.x), so that stretches of large values are spread over all CTAs.  u_slots: row
-// slots of shared memory that receive eps and then hold u (the last u_slots rows of a CTA stay
-// on chip); table_rows: the largest number of rows any CTA owns (entries of the maximum table).
-// predict: count during phase A against predicted thresholds (the vector must have at least 32
-// float4); bar_target: arrivals a grid barrier waits for (the grid size; a test may ask for more
-// to see the bounded waits run out).  spart: two double2 per CTA.  rowcnt: one word per row.
-// Shared memory: [ring of kRing rows][u_slots rows][table of table_rows x 32 uint16].
+// Up to kGroupRows of this warp's cells (local rows) that meet a condition, from row `cursor`
+// on: their rows go to qrow[0 ..), the cursor moves past the last one taken.  Called by all
+// lanes of a warp; returns the number of rows gathered.
+enum GatherWhat { kGatherFlagged, kGatherPending, kGatherNonZero };
+constexpr unsigned short kPending = 0xffffu;   // phase C: the cell qualifies, its count is still to come
+template <GatherWhat WHAT>
+__device__ __forceinline__ int gather_cells(const unsigned short* table, const int nrows, int& cursor,
+                                            unsigned short* qrow, const unsigned int above = 0u) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int n = 0;
+    while (n < kGroupRows && cursor < nrows) {
+        const int r = cursor + lane;
+        unsigned int e = 0u;
+        if (r < nrows) e = table[r * kFusedWarps + w];
+        // (flagged cells only count when their maximum reaches the lowest threshold of interest)
+        const bool hit = WHAT == kGatherFlagged ? (e & kFlagBit) != 0u && (e & kMaxMask) > above
+                         : WHAT == kGatherPending ? e == kPending : e != 0u;
+        unsigned int b = __ballot_sync(0xffffffffu, hit);
+        while (b && n < kGroupRows) {
+            const int bit = __ffs(b) - 1;
+            if (lane == 0) qrow[n] = (unsigned short)(cursor + bit);
+            ++n;
+            b &= b - 1u;
+        }
+        if (b) { cursor += __ffs(b) - 1; break; }
+        cursor += 32;
+    }
+    __syncwarp();
+    return n;
+}
+
+// The sample of one CTA: warp w reads block (c * 32 + w) of G * 32 blocks of 32 float4 spread
+// evenly over the vector.  They are read with plain loads before anything else (so that no row
+// has been overwritten yet) and parked in two ring slots that phase A does not use once the
+// first row has been worked on.
+// Nothing here synchronises a CTA or the grid, and nothing waits for memory to settle (a fence
+// in a warp that streams rows stalls it for microseconds): every warp leaves the power sums of
+// its block's (u - pv) in a slot of shared memory; the warp that comes last adds the 32 slots
+// and adds the CTA's sums to four global accumulators, then one to a count, with plain atomics.
+// Warp 0 of every CTA reads the accumulators and the count once per row (one sector, issued
+// before the row and looked at after it); when the count is complete it forms the bands and
+// hands them to its CTA's warps, which change over at their next row.
+// The prediction only decides where a cell is counted, never what the count is: sums that are
+// incomplete because the count overtook them, or a sample that misleads, give bands that are
+// found out when the exact thresholds are known, and the CTA then counts in full.  (For the
+// same reason it does no harm that the sums are added in the order of arrival, or that another
+// CTA may already have replaced eps by u in a block of the first rows.)
+// This thread's float4 of its warp's sample block: block (c * 32 + w) of G * 32 blocks of 32
+// float4 spread evenly over the whole vector (leaving a stretch out would bias the prediction
+// on vectors whose loud layers are few).
+__device__ __forceinline__ int64_t sample_at(const int64_t n4) {
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int64_t nblk = n4 >> 5;
+    const int64_t blk = (((int64_t)blockIdx.x * kFusedWarps + w) * nblk) / ((int64_t)gridDim.x * kFusedWarps);
+    return (blk << 5) + lane;
+}
+// Called by whole warps, each once.  Out of line: its temporaries are its own.
 template <bool ACC>
-__global__ void __launch_bounds__(kFusedThreads, 1)
-k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, double z,
-           int n_rows, int u_slots, int table_rows, int predict, unsigned int bar_target, Ctrl* __restrict__ ctrl,
-           double2* __restrict__ partials, double2* __restrict__ spart, unsigned int* __restrict__ bars,
-           unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
-           int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
-    // 1 KB alignment keeps every warp's 512 bytes of a row within four 128-byte lines of shared
-    // memory, whatever the size of the static part
-    extern __shared__ __align__(1024) float4 smem4[];
-    __shared__ FusedShared sh;
-    float4* gring = smem4;                                   // kRing x kRowF4 (phase A uses kStages of them)
-    float4* uslot = smem4 + (size_t)kRing * kRowF4;          // u_slots x kRowF4
-    unsigned short* table = reinterpret_cast<unsigned short*>(smem4 + (size_t)(kRing + u_slots) * kRowF4);
+__device__ __noinline__ void publish_sample(const float4* gring, double pv, FusedShared* shp, unsigned int* bars) {
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    float4 a = gring[(size_t)kStages * kRowF4 + tid];
+    if (ACC) {
+        const float4 b = gring[(size_t)(kStages + 1) * kRowF4 + tid];
+        a = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+    }
+    const double x[4] = {(double)a.x - pv, (double)a.y - pv, (double)a.z - pv, (double)a.w - pv};
+    double p1 = 0.0, p2 = 0.0, p3 = 0.0, p4 = 0.0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const double y = x[t] * x[t];
+        p1 += x[t]; p2 += y; p3 = fma(y, x[t], p3); p4 = fma(y, y, p4);
+    }
+    p1 = warp_sum(p1); p2 = warp_sum(p2); p3 = warp_sum(p3); p4 = warp_sum(p4);
+    // the slots borrow an array that only phase C uses
+    double2* slots = reinterpret_cast<double2*>(shp->roundtot);
+    unsigned int before = 0u;
+    if (lane == 0) {
+        slots[2 * w] = make_double2(p1, p2);
+        slots[2 * w + 1] = make_double2(p3, p4);
+        __threadfence_block();
+        before = atomicAdd(&shp->samp_n, 1u);
+    }
+    if (__shfl_sync(0xffffffffu, before, 0) != kFusedWarps - 1) return;
+    // all warps are in: the CTA's sums (slot order, then a shuffle tree) join the global ones
+    __threadfence_block();
+    const volatile double* sv = reinterpret_cast<const volatile double*>(slots);
+    p1 = warp_sum(sv[4 * lane]); p2 = warp_sum(sv[4 * lane + 1]);
+    p3 = warp_sum(sv[4 * lane + 2]); p4 = warp_sum(sv[4 * lane + 3]);
+    if (lane == 0) {
+        double* acc = reinterpret_cast<double*>(bars + kBarSample);
+        atomicAdd(acc + 0, p1); atomicAdd(acc + 1, p2); atomicAdd(acc + 2, p3); atomicAdd(acc + 3, p4);
+        atomicAdd(bars + kBarSample + 8, 1u);
+    }
+}
+
+// What a thread needs to know about its CTA's share of the vector, derived from the launch
+// parameters alone, so that every phase can form it for itself.  Local row r of CTA c is row
+// c + r * G of the vector; only the last row of the vector can be short, and it is the last
+// local row of the CTA that owns it.
+struct Rows {
+    int nrows;          // rows of this CTA
+    int first_kept;     // rows from here on stay on chip after phase A (the short last row of the
+                        // vector, if this CTA owns it, is among them: u_slots >= 1)
+    int64_t n4;         // float4 in the vector
+    int64_t stride4;    // from a local row to the next
+    int64_t first4;     // this thread's float4 in local row 0
+    int64_t tail_i;     // this lane's element of the ragged tail (d mod 4 elements)
+    bool in_last_row;   // this thread has a float4 in the CTA's last row
+    bool owns_tail;     // this thread holds an element of the ragged tail
+};
+__device__ __forceinline__ Rows rows_of(const int64_t d, const int n_rows, const int u_slots) {
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int c = blockIdx.x, G = gridDim.x;
-    const int64_t n4 = d >> 2;
+    Rows q;
+    q.n4 = d >> 2;
+    q.nrows = c < n_rows ? (n_rows - c + G - 1) / G : 0;
+    q.stride4 = (int64_t)G * kRowF4;
+    q.first4 = (int64_t)c * kRowF4 + tid;
+    const bool has_last = q.nrows > 0 && (c + (q.nrows - 1) * G == n_rows - 1);
+    q.in_last_row = !(has_last && (q.n4 & (kRowF4 - 1)) != 0) || tid < (int)(q.n4 & (kRowF4 - 1));
+    q.first_kept = q.nrows > u_slots ? q.nrows - u_slots : 0;
+    q.owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
+    q.tail_i = (q.n4 << 2) + lane;
+    return q;
+}
 
-    // this CTA's rows: local row r is row c + r * G of the vector; only the last row of the
-    // vector can be short, and it is the last local row of the CTA that owns it
-    const int nrows = c < n_rows ? (n_rows - c + G - 1) / G : 0;
-    const int64_t stride4 = (int64_t)G * kRowF4;             // from a local row to the next
-    const int64_t first4 = (int64_t)c * kRowF4 + tid;        // this thread's float4 in local row 0
-    const bool has_last = nrows > 0 && (c + (nrows - 1) * G == n_rows - 1);
-    const bool in_last_row = !(has_last && (n4 & (kRowF4 - 1)) != 0) || tid < (int)(n4 & (kRowF4 - 1));
-    // rows from first_kept on stay on chip after phase A; the short last row of the vector, if
-    // this CTA owns it, is its last row and therefore among them (u_slots >= 1)
-    const int first_kept = nrows > u_slots ? nrows - u_slots : 0;
-    const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
-    const int64_t tail_i = (n4 << 2) + lane;
-    const float4* g4 = reinterpret_cast<const float4*>(src);
-    float4* e4 = reinterpret_cast<float4*>(eps);
-    // where u is read again after phase A: eps holds it for the sparsifier, the input itself otherwise
-    const float* uvec = ACC ? eps : src;
+// Shared memory of the kernel: [FusedShared, kFusedStaticBytes][ring of kRing rows][u_slots rows]
+// [table of table_rows x 32 uint16].  The rows start on a 1 KB boundary, which keeps every
+// warp's 512 bytes of a row within four 128-byte lines.
+struct Smem {
+    FusedShared* sh;
+    float4* gring;           // kRing x kRowF4 (phase A uses kStages of them for g)
+    float4* uslot;           // u_slots x kRowF4
+    unsigned short* table;   // one entry per (local row, warp)
+};
+__device__ __forceinline__ Smem smem_of(const int u_slots) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    Smem m;
+    m.sh = reinterpret_cast<FusedShared*>(smem_raw);
+    float4* rows = reinterpret_cast<float4*>(smem_raw + kFusedStaticBytes);
+    m.gring = rows;
+    m.uslot = rows + (size_t)kRing * kRowF4;
+    m.table = reinterpret_cast<unsigned short*>(rows + (size_t)(kRing + u_slots) * kRowF4);
+    return m;
+}
+#define GK_FUSED_VIEW(d, n_rows, u_slots)                                               \
+    const Rows rows_ = rows_of(d, n_rows, u_slots);                                     \
+    const Smem smem_ = smem_of(u_slots);                                                \
+    FusedShared& sh = *smem_.sh;                                                        \
+    float4* const gring = smem_.gring; float4* const uslot = smem_.uslot;               \
+    unsigned short* const table = smem_.table;                                          \
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;                         \
+    const int c = blockIdx.x, G = gridDim.x;                                            \
+    const int nrows = rows_.nrows, first_kept = rows_.first_kept;                       \
+    const int64_t n4 = rows_.n4, stride4 = rows_.stride4, first4 = rows_.first4, tail_i = rows_.tail_i; \
+    const bool in_last_row = rows_.in_last_row, owns_tail = rows_.owns_tail;            \
+    (void)gring; (void)uslot; (void)table; (void)lane; (void)w; (void)c; (void)G; (void)nrows; (void)first_kept; \
+    (void)n4; (void)stride4; (void)first4; (void)tail_i; (void)in_last_row; (void)owns_tail; (void)sh
+
+// Phase B, the short way: the six upper candidates over the cells that phase A left (flagged),
+// added to phase A's own counts (pacc, two candidates to a float).  The cells are few and
+// scattered, so every warp gathers its own eight at a time and loads them together, from shared
+// memory where the row is on chip, else from L2.  Leaves the CTA's counts in sh.cta_counts.
+// Out of line: its registers are its own.
+__device__ __noinline__ void count_short_way(const float* __restrict__ uvec, const int64_t d, const int n_rows,
+                                             const int u_slots, const float pacc0, const float pacc1,
+                                             const float pacc2, const float tail_u, unsigned int* __restrict__ bars) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
     const float4* u4 = reinterpret_cast<const float4*>(uvec);
-    float tail_u = 0.f;
-    const bool wide_ok = ACC && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
-    unsigned int* tot0 = bars + kBarTotals;               // global counts of the first count
-    unsigned int* tot1 = bars + kBarTotals + kNumCand;    // ... of the second, full one
-    if (c == 0 && tid == 0) {
-        ctrl->stats.status = GK_DEV_OK;
-        ctrl->phase_t[0] = global_timer_ns();
+    const float pacc[kUpper / 2] = {pacc0, pacc1, pacc2};
+    float cs[kUpper], acc[kUpper];
+#pragma unroll
+    for (int j = 0; j < kUpper; ++j) cs[j] = sh.cand32[cand_by_factor(kNumCand - kUpper + j)];
+#pragma unroll
+    for (int j = 0; j < kUpper / 2; ++j) {
+        const float hi = floorf(pacc[j] * (1.0f / kPackScale));
+        acc[2 * j] = pacc[j] - hi * kPackScale;
+        acc[2 * j + 1] = hi;
     }
-    // optional per-CTA trace: start, before / after each barrier, end
+    const unsigned int t0 = __float_as_uint(cs[0]) >> 16, t1 = __float_as_uint(cs[1]) >> 16,
+                       t3 = __float_as_uint(cs[3]) >> 16;
+    auto count_upper = [&](const float4 x, const unsigned int rm) {   // rm > t0
+        const float a0 = fabsf(x.x), a1 = fabsf(x.y), a2 = fabsf(x.z), a3 = fabsf(x.w);
+        count_tier<0, 1>(a0, a1, a2, a3, cs, acc);
+        if (rm > t1) {
+            count_tier<1, 3>(a0, a1, a2, a3, cs, acc);
+            if (rm > t3) count_tier<3, kUpper>(a0, a1, a2, a3, cs, acc);
+        }
+    };
+    unsigned int n_left = 0u;   // cells this warp had left
+    for (int cursor = 0; cursor < nrows;) {
+        const int n = gather_cells<kGatherFlagged>(table, nrows, cursor, sh.qrow[w], t0);
+        n_left += (unsigned int)n;
+        float4 v[kGroupRows];
+#pragma unroll
+        for (int q = 0; q < kGroupRows; ++q) {
+            v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (q < n) {
+                const int r = sh.qrow[w][q];
+                const int64_t i = first4 + (int64_t)r * stride4;
+                if (i < n4) v[q] = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(u4 + i);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kGroupRows; ++q) {
+            if (q < n) {
+                count_upper(v[q], (unsigned int)table[sh.qrow[w][q] * kFusedWarps + w] & kMaxMask);
+            }
+        }
+        __syncwarp();
+    }
+    if (owns_tail) {
+        const float a = fabsf(tail_u);
+#pragma unroll
+        for (int j = 0; j < kUpper; ++j) acc[j] += gt_as_float(a, cs[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < kUpper; ++j) {
+        const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+        if (lane == 0 && ws) atomicAdd(&sh.cta_counts[cand_by_factor(kNumCand - kUpper + j)], ws);
+    }
+    if (lane == 0 && n_left) atomicAdd(&bars[kBarInfo + 3], n_left);
+    __syncthreads();
+}
+
+// Phase B in full: all ten candidates over all cells of this CTA.  Leaves the CTA's counts in
+// sh.cta_counts (cleared first when `again`: a second count after the short way).
+__device__ __noinline__ void count_in_full(const float* __restrict__ uvec, const int64_t d, const int n_rows,
+                                           const int u_slots, const float tail_u, const bool again) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
+    const float4* u4 = reinterpret_cast<const float4*>(uvec);
+    // candidates in ascending order of value; cs[j] = value, sh.order[j] = its index
+    float cs[kNumCand], acc[kNumCand];
+#pragma unroll
+    for (int j = 0; j < kNumCand; ++j) { cs[j] = sh.cand32[sh.order[j]]; acc[j] = 0.f; }
+    // tier limits: top 16 bits of the tier's lowest candidate, rounded down; a negative
+    // candidate is exceeded by everything, and candidates ascend, so testing the lowest suffices
+    const Tiers tier = make_tiers(cs);
+    const unsigned int always = 0x10000u;  // above every 16-bit maximum
+    const bool any_neg = cs[0] < 0.f;
+    const unsigned short* trow = table + w;
+    auto row_max = [&](int r) -> unsigned int {
+        return any_neg ? always : ((unsigned int)trow[r * kFusedWarps] & kMaxMask);
+    };
+    // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
+    // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows.  They are
+    // taken from the last written to the first: the rows written last are the ones most
+    // likely still in L2, and reading them first keeps the misses on the oldest rows from
+    // pushing them out before their turn.
+    int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;  // the row the next fetch brings in
+    auto fetch_u = [&](int q) {   // q-th row in this order: local row first_kept - 1 - q
+        if (q < first_kept) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, u4 + fo);
+        cp_async_commit();
+        fo -= stride4;
+    };
+#pragma unroll
+    for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
+    static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
+#pragma unroll 2
+    for (int q = 0; q < first_kept; ++q) {
+        fetch_u(q + kRing - 1);
+        cp_async_wait<kRing - 1>();
+        count_float4(gring[((q & (kRing - 1)) << 10) + tid], row_max(first_kept - 1 - q), cs, tier, acc);
+    }
+    cp_async_wait<0>();
+    for (int r = first_kept; r < nrows; ++r) {
+        if (r != nrows - 1 || in_last_row)
+            count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], row_max(r), cs, tier, acc);
+    }
+    if (owns_tail) {
+        const float a = fabsf(tail_u);
+#pragma unroll
+        for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
+    }
+    if (again) {
+        __syncthreads();   // the first count's sums have been read by everyone
+        if (tid < kNumCand) sh.cta_counts[tid] = 0u;
+        __syncthreads();
+    }
+#pragma unroll
+    for (int j = 0; j < kNumCand; ++j) {
+        const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+        if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
+    }
+    __syncthreads();
+}
+
+// Phase C: the survivors |u_i| > threshold of this CTA's rows, counted per cell, the per-row
+// totals exchanged through one more grid barrier, then written as ordered pairs (and their
+// slots of eps cleared, ACC).  Returns false when the barrier's bounded wait ran out.
+template <bool ACC>
+__device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, float* __restrict__ eps, const int64_t d,
+                                               const int n_rows, const int u_slots, const unsigned int bar_target,
+                                               unsigned int* __restrict__ bars, unsigned int* __restrict__ rowcnt,
+                                               int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+                                               const int64_t cap, const float tail_u,
+                                               unsigned long long* __restrict__ trace) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
+    const float4* u4 = reinterpret_cast<const float4*>(uvec);
     auto stamp = [&](int slot) {
         if (trace != nullptr && tid == 0) trace[(size_t)c * kTraceSlots + slot] = global_timer_ns();
     };
-    stamp(0);
-
-    // phase A's counts of the six upper candidates over the cells it settled, and whether this
-    // CTA holds a prediction
-    float pacc[kUpper];
-#pragma unroll
-    for (int j = 0; j < kUpper; ++j) pacc[j] = 0.f;
-    bool pred_live = false;
-
-    // ------------------------------------------------------------------ phase A
     {
-        const double pv = (double)src[0];
-        double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
-        // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
-        // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
-        // The operator form has one operand, which takes the way of eps.
-        int64_t fi = first4;  // the row the next fetch brings in
-        // Where the eps of local row r lands.  Normally the slot that will hold u.  A CTA with so
-        // many rows that its table leaves fewer slots than rows in flight takes eps through the
-        // half of the ring that g does not use, and only its last rows are kept on chip.
-        const bool eps_ring = u_slots < kStages;
-        auto eps_slot = [&](int r) -> float4* {
-            return eps_ring ? gring + (size_t)(kStages + r % kStages) * kRowF4 : uslot + (size_t)(r % u_slots) * kRowF4;
-        };
-        auto fetch = [&](int r) {
-            if (r < nrows && fi < n4) {
-                if (ACC) {
-                    cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
-                    cp_async16(eps_slot(r) + tid, e4 + fi);
-                } else {
-                    cp_async16(eps_slot(r) + tid, g4 + fi);
-                }
-            }
-            cp_async_commit();
-            fi += stride4;
-        };
-#pragma unroll
-        for (int r = 0; r < kStages - 1; ++r) fetch(r);
-
-        // The sample: warp w of CTA c reads block (c * 32 + w) of G * 32 blocks of 32 float4 spread
-        // evenly over the vector, and the CTA publishes the power sums of (u - pv).  (Another CTA
-        // may already have replaced eps by u in a block of the first rows; the sample then sees
-        // g + u there.  That can only cost accuracy of the prediction, never of the result.)
-        int pred_state = 0;   // 1: sample published, totals not yet seen
-        if (predict) {
-            const int64_t nblk = n4 >> 5;
-            const int64_t blk = (((int64_t)c * kFusedWarps + w) * nblk) / ((int64_t)G * kFusedWarps);
-            const int64_t at = (blk << 5) + lane;
-            float4 a = __ldcg(g4 + at);
-            if (ACC) {
-                const float4 b = __ldcg(e4 + at);
-                a = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
-            }
-            const double x[4] = {(double)a.x - pv, (double)a.y - pv, (double)a.z - pv, (double)a.w - pv};
-            double p1 = 0.0, p2 = 0.0, p3 = 0.0, p4 = 0.0;
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const double y = x[t] * x[t];
-                p1 += x[t]; p2 += y; p3 = fma(y, x[t], p3); p4 = fma(y, y, p4);
-            }
-            const double2 a12 = block_sum2<kFusedThreads>(p1, p2, sh.red);
-            const double2 a34 = block_sum2<kFusedThreads>(p3, p4, sh.red);
-            if (tid == 0) {
-                spart[2 * c] = a12;
-                spart[2 * c + 1] = a34;
-                __threadfence();
-                atomicAdd(&bars[kBarPublished], 1u);
-            }
-            pred_state = 1;
-        }
-        unsigned int ptl0 = 0u, ptl1 = 0u, ptl3 = 0u;   // tier limits of the predicted bands
-        unsigned int n_left = 0u;                        // cells of this warp left to phase B
-        const int poll_end = nrows / 3;                  // a prediction that comes later is not worth having
-
-        int64_t i = first4;
-        for (int r = 0; r < nrows; ++r, i += stride4) {
-            if (pred_state == 1 && r >= kPredPollFirst) {
-                // have all CTAs published?  One look per row; the answer goes through shared memory
-                // (two words in turn, so that a thread still reading last row's cannot see this row's)
-                if (tid == 0) sh.poll[r & 1] = ld_acquire_u32(&bars[kBarPublished]) >= (unsigned)G ? 1 : 0;
-                __syncthreads();
-                if (sh.poll[r & 1]) {
-                    double a1 = 0.0, a2 = 0.0, a3 = 0.0, a4 = 0.0;
-                    for (int t = tid; t < G; t += kFusedThreads) {
-                        const double2 p = __ldcg(&spart[2 * t]), q = __ldcg(&spart[2 * t + 1]);
-                        a1 += p.x; a2 += p.y; a3 += q.x; a4 += q.y;
-                    }
-                    const double2 t12 = block_sum2<kFusedThreads>(a1, a2, sh.red);
-                    const double2 t34 = block_sum2<kFusedThreads>(a3, a4, sh.red);
-                    if (tid == 0)
-                        sh.pred_ok = predict_bands(t12.x, t12.y, t34.x, t34.y, (double)G * kSampleElems, pv, z,
-                                                   sh.plo, sh.phi) ? 1 : 0;
-                    __syncthreads();
-                    pred_state = 0;
-                    if (sh.pred_ok) {
-                        pred_live = true;
-                        // top 16 bits of each tier's lowest band edge, rounded down (the edges are positive)
-                        ptl0 = __float_as_uint(sh.plo[0]) >> 16;
-                        ptl1 = __float_as_uint(sh.plo[1]) >> 16;
-                        ptl3 = __float_as_uint(sh.plo[3]) >> 16;
-                    }
-                } else if (r >= poll_end) {
-                    pred_state = 0;
-                }
-            }
-            fetch(r + kStages - 1);
-            cp_async_wait<kStages - 1>();
-            const bool one = i < n4;
-            float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (one) {
-                float4* es = eps_slot(r) + tid;
-                if (ACC) {
-                    const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *es;
-                    u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
-                    if (!eps_ring) *es = u0;
-                } else {
-                    u0 = *es;
-                }
-                if (eps_ring && r >= first_kept) uslot[(size_t)(r % u_slots) * kRowF4 + tid] = u0;
-                const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
-                             x3 = (double)u0.w - pv;
-                s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
-                s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
-            }
-            // u goes out in 32-byte stores by the even lanes (own float4 and the right neighbour's),
-            // marked to stay in L2: the next two phases read most of u again
-            if (ACC) {
-                float4 nb;
-                nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
-                nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
-                const bool pair = wide_ok && (i + 1 < n4);  // this lane and its right neighbour are in range
-                if ((lane & 1) == 0) {
-                    if (pair) st_keep32(e4 + i, u0, nb);
-                    else if (one) e4[i] = u0;
-                } else if (one && !wide_ok) {
-                    e4[i] = u0;
-                }
-            }
-            // largest magnitude of each (row, warp) cell, top 16 bits rounded up (15 bits for
-            // finite values), and above it the flag "not settled here"
-            const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
-            unsigned int entry = (m0 + 0xffffu) >> 16;
-            if (predict) {
-                if (!pred_live) {
-                    entry |= kFlagBit;
-                } else if (entry > ptl0) {
-                    // the cell can reach the lowest band: per candidate the elements above the band's
-                    // upper edge, and over all candidates those above the lower edges; the two sums
-                    // differ exactly when an element lies inside a band
-                    const float a0 = fabsf(u0.x), a1 = fabsf(u0.y), a2 = fabsf(u0.z), a3 = fabsf(u0.w);
-                    float h[kUpper];
-#pragma unroll
-                    for (int j = 0; j < kUpper; ++j) h[j] = 0.f;
-                    float below = 0.f;
-                    auto band = [&](const int j) {
-                        const float lo = sh.plo[j], hi = sh.phi[j];
-                        h[j] = (gt_as_float(a0, hi) + gt_as_float(a1, hi)) + (gt_as_float(a2, hi) + gt_as_float(a3, hi));
-                        below += (gt_as_float(a0, lo) + gt_as_float(a1, lo)) + (gt_as_float(a2, lo) + gt_as_float(a3, lo));
-                    };
-                    band(0);
-                    if (entry > ptl1) {
-                        band(1); band(2);
-                        if (entry > ptl3) { band(3); band(4); band(5); }
-                    }
-                    const float above = ((h[0] + h[1]) + (h[2] + h[3])) + (h[4] + h[5]);
-                    if (__any_sync(0xffffffffu, below != above)) {
-                        entry |= kFlagBit;
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < kUpper; ++j) pacc[j] += h[j];
-                    }
-                }
-            }
-            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)entry;
-            n_left += (entry >> 15);
-        }
-        if (pred_live && lane == 0 && n_left) atomicAdd(&bars[kBarInfo + 3], n_left);
-        if (pred_live && tid == 0) atomicAdd(&bars[kBarInfo + 0], 1u);
-        cp_async_wait<0>();
-        if (owns_tail) {
-            tail_u = ACC ? src[tail_i] + eps[tail_i] : src[tail_i];
-            if (ACC) eps[tail_i] = tail_u;
-            const double x = (double)tail_u - pv;
-            s0 += x; q0 = fma(x, x, q0);
-        }
-        const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
-        if (tid == 0) partials[c] = part;
-        stamp(1);
-        if (!grid_barrier(&bars[kBarStats], bar_target, &sh.ok)) {
-            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
-            goto leave;
-        }
-        stamp(2);
-        // every CTA forms the same totals: thread t takes partial t, t + T, ...
-        double s = 0.0, q = 0.0;
-        for (int t = tid; t < G; t += kFusedThreads) {
-            const double2 p = __ldcg(&partials[t]);
-            s += p.x; q += p.y;
-        }
-        const double2 tot = block_sum2<kFusedThreads>(s, q, sh.red);
-        if (tid == 0) {
-            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
-            alg1_thresholds(st, tot.x, tot.y, pv, d, k, z);
-            // candidate indices in ascending order of threshold
-            const bool neg = sh.stats.thres0 < 0.0;
-#pragma unroll
-            for (int j = 0; j < kNumCand; ++j) sh.order[j] = cand_ascending(j, neg);
-            // phase A's counts stand if every exact candidate lies within its predicted band
-            bool fast = pred_live && sh.stats.thres0 > 0.0;
-            if (fast) {
-#pragma unroll
-                for (int j = 0; j < kUpper; ++j) {
-                    const float cj = sh.cand32[cand_by_factor(kNumCand - kUpper + j)];
-                    fast = fast && sh.plo[j] <= cj && cj <= sh.phi[j];
-                }
-            }
-            sh.fast = fast ? 1 : 0;
-            sh.recount = 0;
-        }
-        if (tid < kNumCand) sh.cta_counts[tid] = 0u;
-        if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
-        __syncthreads();
-    }
-
-    // ------------------------------------------------------------------ phase B and the rounds
-    // First count: the short way where this CTA's prediction held, else in full.  If the rounds
-    // then ask for a candidate that some CTA left out, the CTAs that took the short way count
-    // again in full and the sums are formed a second time.
-    for (int pass = 0; pass < 2; ++pass) {
-        const bool fast = pass == 0 && sh.fast != 0;
-        if (pass == 0 || sh.fast != 0) {
-            // candidates in ascending order of value; cs[j] = value, sh.order[j] = its index
-            float cs[kNumCand], acc[kNumCand];
-#pragma unroll
-            for (int j = 0; j < kNumCand; ++j) {
-                cs[j] = sh.cand32[sh.order[j]];
-                acc[j] = (fast && j >= kNumCand - kUpper) ? pacc[j - (kNumCand - kUpper)] : 0.f;
-            }
-            // tier limits: top 16 bits of the tier's lowest candidate, rounded down; a negative
-            // candidate is exceeded by everything, and candidates ascend, so testing the lowest suffices
-            Tiers tier = make_tiers(cs);
-            if (fast) tier.t0 = __float_as_uint(cs[kNumCand - kUpper]) >> 16;   // the short way starts at 3/4 thres0 (> 0)
-            const unsigned int always = 0x10000u;  // above every 16-bit maximum
-            const bool any_neg = cs[0] < 0.f;
-            const unsigned short* trow = table + w;
-            // is the cell of local row r to be counted now, and with which maximum
-            auto wanted = [&](int r) -> bool { return !fast || (trow[r * kFusedWarps] & kFlagBit) != 0u; };
-            auto row_max = [&](int r) -> unsigned int {
-                return any_neg ? always : ((unsigned int)trow[r * kFusedWarps] & kMaxMask);
-            };
-            auto count_cell = [&](const float4 x, const int r) {
-                if (fast) count_float4<kNumCand - kUpper>(x, row_max(r), cs, tier, acc);
-                else count_float4<0>(x, row_max(r), cs, tier, acc);
-            };
-            // rows that are not on chip come back from eps (L2 / HBM) through the ring that carried g
-            // in phase A, kRing - 1 rows ahead of the counting; all of them are full rows.  They are
-            // taken from the last written to the first: the rows written last are the ones most
-            // likely still in L2, and reading them first keeps the misses on the oldest rows from
-            // pushing them out before their turn.
-            int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;  // the row the next fetch brings in
-            auto fetch_u = [&](int q) {   // q-th row in this order: local row first_kept - 1 - q
-                if (q < first_kept && wanted(first_kept - 1 - q)) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, u4 + fo);
-                cp_async_commit();
-                fo -= stride4;
-            };
-#pragma unroll
-            for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
-            static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
-#pragma unroll 2
-            for (int q = 0; q < first_kept; ++q) {
-                fetch_u(q + kRing - 1);
-                cp_async_wait<kRing - 1>();
-                const int r = first_kept - 1 - q;
-                if (wanted(r)) count_cell(gring[((q & (kRing - 1)) << 10) + tid], r);
-            }
-            cp_async_wait<0>();
-            for (int r = first_kept; r < nrows; ++r) {
-                if ((r != nrows - 1 || in_last_row) && wanted(r))
-                    count_cell(uslot[(size_t)(r % u_slots) * kRowF4 + tid], r);
-            }
-            if (owns_tail) {
-                const float a = fabsf(tail_u);
-#pragma unroll
-                for (int j = 0; j < kNumCand; ++j) acc[j] += gt_as_float(a, cs[j]);
-            }
-            if (pass == 1) {
-                __syncthreads();   // the first count's sums have been read by everyone
-                if (tid < kNumCand) sh.cta_counts[tid] = 0u;
-                __syncthreads();
-            }
-#pragma unroll
-            for (int j = 0; j < kNumCand; ++j) {
-                const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
-                if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
-            }
-            __syncthreads();
-        }
-        // this CTA's counts join the global sums; the short way leaves the four lower candidates out
-        if (tid < kNumCand) {
-            const unsigned int v = sh.cta_counts[tid];
-            if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
-        }
-        if (fast && tid == 0) {
-            atomicOr(&bars[kBarInvalid], kLowCandMask);
-            atomicAdd(&bars[kBarInfo + 1], 1u);
-        }
-        if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
-        stamp(3);
-        if (!grid_barrier(&bars[pass == 0 ? kBarCounts : kBarCounts2], bar_target, &sh.ok)) {
-            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
-            goto leave;
-        }
-        if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
-        stamp(4);
-
-        // -------------------------------------------------------------- the rounds
-        if (tid < kNumCand) sh.col[tid] = (unsigned long long)ld_acquire_u32((pass == 0 ? tot0 : tot1) + tid);
-        __syncthreads();
-        if (tid == 0) {
-            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
-            unsigned int visited = 0u;
-            sh.chosen = alg1_resolve(st, k, &visited);
-            sh.n_staged = 0u;
-            // a candidate the rounds evaluated but some CTA did not count: count again, in full
-            sh.recount = (pass == 0 && (visited & ld_acquire_u32(&bars[kBarInvalid])) != 0u) ? 1 : 0;
-        }
-        __syncthreads();
-        if (!sh.recount) break;
-        if (c == 0 && tid == 0) bars[kBarInfo + 2] = 1u;
-    }
-    if (c == 0 && tid == 0) {
-        const long long all = sh.stats.nnz;
-        const long long written = all < cap ? all : cap;
-        // every field but the status word, which was cleared at the start and only ever has
-        // flags added to it (a CTA that gave up waiting may have added one already)
-        gk_stats* o = &ctrl->stats;
-        o->mu = sh.stats.mu; o->sigma = sh.stats.sigma; o->z = sh.stats.z;
-        o->thres0 = sh.stats.thres0; o->thr_final = sh.stats.thr_final;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) o->counts[j] = sh.stats.counts[j];
-        o->rounds = sh.stats.rounds; o->nnz = all; o->emitted = written;
-        const int flags = sh.stats.status | (all > cap ? GK_DEV_TRUNCATED : 0);
-        if (flags) atomicOr(&o->status, flags);
-        *nnz_out = written;
-        ctrl->phase_t[4] = global_timer_ns();
-    }
-
-    // ------------------------------------------------------------------ phase C
-    // The survivor count of the whole vector is known to every CTA; with none there is nothing
-    // left to do (the same decision in every CTA, so the barrier below is reached by all or none).
-    if (sh.stats.nnz != 0) {
         const float thr = sh.thr_sel;
         const unsigned int mine = sh.cta_counts[sh.chosen];  // survivors in this CTA's rows
         // a segment can hold a survivor only if its recorded maximum (rounded up to 16 bits)
         // exceeds the threshold's top 16 bits; a negative threshold admits everything
         const bool all_pass = thr < 0.0f;
         const unsigned int thr16 = __float_as_uint(fmaxf(thr, 0.0f)) >> 16;
-        constexpr unsigned short kPending = 0xffffu;
-        // up to kGroupRows rows of this warp whose entry is pending (want_pending) or non-zero,
-        // from `cursor` on
-        auto gather = [&](int& cursor, const bool want_pending) -> int {
-            int n = 0;
-            while (n < kGroupRows && cursor < nrows) {
-                const int r = cursor + lane;
-                unsigned int e = 0u;
-                if (r < nrows) e = table[r * kFusedWarps + w];   // a count by now, or the pending mark
-                const bool hit = want_pending ? (e == kPending) : (e != 0u);
-                unsigned int b = __ballot_sync(0xffffffffu, hit);
-                while (b && n < kGroupRows) {
-                    const int bit = __ffs(b) - 1;
-                    if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
-                    ++n;
-                    b &= b - 1u;
-                }
-                if (b) { cursor += __ffs(b) - 1; break; }
-                cursor += 32;
-            }
-            __syncwarp();
-            return n;
-        };
         auto load_row = [&](int r, int64_t i) -> float4 {
             return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(u4 + i);
         };
@@ -682,7 +573,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             } else {
                 // few qualifying segments: they are gathered eight at a time so that their loads overlap
                 for (int cursor = 0; cursor < nrows;) {
-                    const int n = gather(cursor, true);
+                    const int n = gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w]);
                     float4 v[kGroupRows];
 #pragma unroll
                     for (int q = 0; q < kGroupRows; ++q) {
@@ -735,8 +626,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         }
         stamp(5);
         if (!grid_barrier(&bars[kBarRows], bar_target, &sh.ok)) {
-            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
-            goto leave;
+            return false;
         }
         stamp(6);
         if (mine != 0u) {
@@ -801,7 +691,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             } else
             // step 3: every warp writes the survivors of its segments that have any
             for (int cursor = 0; cursor < nrows;) {
-                const int n = gather(cursor, false);
+                const int n = gather_cells<kGatherNonZero>(table, nrows, cursor, sh.qrow[w]);
                 float4 v[kGroupRows];
 #pragma unroll
                 for (int q = 0; q < kGroupRows; ++q) {
@@ -863,6 +753,345 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         }
     }
 
+    return true;
+}
+
+// ACC: the sparsifier (src = g, u = g + eps is formed, stored over eps and cleared where
+// selected); !ACC: the operator on a given vector (src = u, read only; eps is not used).
+// n_rows: rows of 1024 float4 in the whole vector; CTA c owns rows c, c + G, c + 2G, ...
+// (G = gridDim.x), so that stretches of large values are spread over all CTAs.  u_slots: row
+// slots of shared memory that receive eps and then hold u (the last u_slots rows of a CTA stay
+// on chip); table_rows: the largest number of rows any CTA owns (entries of the maximum table).
+// PRED: count during phase A against predicted thresholds (the vector must have at least 32
+// float4 and no CTA more than kPredMaxRows rows); bar_target: arrivals a grid barrier waits for (the grid size; a test may ask for more
+// to see the bounded waits run out).  rowcnt: one word per row.
+template <bool ACC, bool PRED>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, double z,
+           int n_rows, int u_slots, int table_rows, unsigned int bar_target, Ctrl* __restrict__ ctrl,
+           double2* __restrict__ partials, unsigned int* __restrict__ bars,
+           unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+           int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
+    const float4* g4 = reinterpret_cast<const float4*>(src);
+    float4* e4 = reinterpret_cast<float4*>(eps);
+    // where u is read again after phase A: eps holds it for the sparsifier, the input itself otherwise
+    const float* uvec = ACC ? eps : src;
+    const float4* u4 = reinterpret_cast<const float4*>(uvec);
+    float tail_u = 0.f;
+    const bool wide_ok = ACC && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
+    unsigned int* tot0 = bars + kBarTotals;               // global counts of the first count
+    unsigned int* tot1 = bars + kBarTotals + kNumCand;    // ... of the second, full one
+    if (c == 0 && tid == 0) {
+        ctrl->stats.status = GK_DEV_OK;
+        ctrl->phase_t[0] = global_timer_ns();
+    }
+    if (PRED) {
+        if (tid == 0) { sh.samp_n = 0u; sh.pred_ready = 0; }
+        __syncthreads();
+    }
+    // optional per-CTA trace: start, before / after each barrier, end
+    auto stamp = [&](int slot) {
+        if (trace != nullptr && tid == 0) trace[(size_t)c * kTraceSlots + slot] = global_timer_ns();
+    };
+    stamp(0);
+
+    // phase A's counts of the six upper candidates over the cells it settled
+    // (two candidates to a float: counts of candidates 2 j and 2 j + 1 as lo + 8192 * hi)
+    float pacc[kUpper / 2];
+#pragma unroll
+    for (int j = 0; j < kUpper / 2; ++j) pacc[j] = 0.f;
+
+    // ------------------------------------------------------------------ phase A
+    {
+        const double pv = (double)src[0];
+        double s0 = 0.0, q0 = 0.0, s1 = 0.0, q1 = 0.0;
+        // rows are fetched kStages - 1 ahead by asynchronous copies: g into a ring, eps into the
+        // slot that will hold u.  Every thread copies and later reads only its own 16 bytes.
+        // The operator form has one operand, which takes the way of eps.
+        int64_t fi = first4;  // the row the next fetch brings in
+        // Where the eps of local row r lands.  Normally the slot that will hold u.  A CTA with so
+        // many rows that its table leaves fewer slots than rows in flight takes eps through the
+        // half of the ring that g does not use, and only its last rows are kept on chip.
+        const bool eps_ring = u_slots < kStages;
+        auto eps_slot = [&](int r) -> float4* {
+            return eps_ring ? gring + (size_t)(kStages + r % kStages) * kRowF4 : uslot + (size_t)(r % u_slots) * kRowF4;
+        };
+        auto fetch = [&](int r) {
+            if (r < nrows && fi < n4) {
+                if (ACC) {
+                    cp_async16(gring + (size_t)(r % kStages) * kRowF4 + tid, g4 + fi);
+                    cp_async16(eps_slot(r) + tid, e4 + fi);
+                } else {
+                    cp_async16(eps_slot(r) + tid, g4 + fi);
+                }
+            }
+            cp_async_commit();
+            fi += stride4;
+        };
+        int pred_state = PRED ? 1 : 0;   // this warp still waits for the predicted bands
+        // the sample's loads go first: they are in flight while the first rows are fetched and are
+        // read (and parked in shared memory) only after row 0
+        float4 sample_g = make_float4(0.f, 0.f, 0.f, 0.f), sample_e = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (PRED) {
+            const int64_t at = sample_at(n4);
+            sample_g = __ldcg(g4 + at);
+            if (ACC) sample_e = __ldcg(e4 + at);
+        }
+#pragma unroll
+        for (int r = 0; r < kStages - 1; ++r) fetch(r);
+        // warp 0, lanes 0..4: the global sample sums (lanes 0..3) and the count of CTAs (lane 4) at its last look
+        unsigned long long seen = 0ull;
+        const unsigned long long* sums = reinterpret_cast<const unsigned long long*>(bars + kBarSample);
+        unsigned int ptl0 = 0u, ptl1 = 0u, ptl3 = 0u;   // tier limits of the predicted bands
+
+        // One row: u = g + eps out to eps and into its slot, the fp64 sums, the cell's table entry.
+        // COUNTING: the prediction is in place and the six upper candidates are counted on the way.
+        auto row_body = [&](const int r, const int64_t i, auto counting) {
+            constexpr bool COUNTING = decltype(counting)::value;
+            fetch(r + kStages - 1);
+            cp_async_wait<kStages - 1>();
+            const bool one = i < n4;
+            float4 u0 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (one) {
+                float4* es = eps_slot(r) + tid;
+                if (ACC) {
+                    const float4 a0 = gring[(size_t)(r % kStages) * kRowF4 + tid], b0 = *es;
+                    u0 = make_float4(a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w);
+                    if (!eps_ring) *es = u0;
+                } else {
+                    u0 = *es;
+                }
+                if (eps_ring && r >= first_kept) uslot[(size_t)(r % u_slots) * kRowF4 + tid] = u0;
+                const double x0 = (double)u0.x - pv, x1 = (double)u0.y - pv, x2 = (double)u0.z - pv,
+                             x3 = (double)u0.w - pv;
+                s0 += x0; q0 = fma(x0, x0, q0); s1 += x1; q1 = fma(x1, x1, q1);
+                s0 += x2; q0 = fma(x2, x2, q0); s1 += x3; q1 = fma(x3, x3, q1);
+            }
+            // u goes out in 32-byte stores by the even lanes (own float4 and the right neighbour's),
+            // marked to stay in L2: the next two phases read most of u again
+            if (ACC) {
+                float4 nb;
+                nb.x = __shfl_down_sync(0xffffffffu, u0.x, 1); nb.y = __shfl_down_sync(0xffffffffu, u0.y, 1);
+                nb.z = __shfl_down_sync(0xffffffffu, u0.z, 1); nb.w = __shfl_down_sync(0xffffffffu, u0.w, 1);
+                const bool pair = wide_ok && (i + 1 < n4);  // this lane and its right neighbour are in range
+                if ((lane & 1) == 0) {
+                    if (pair) st_keep32(e4 + i, u0, nb);
+                    else if (one) e4[i] = u0;
+                } else if (one && !wide_ok) {
+                    e4[i] = u0;
+                }
+            }
+            // largest magnitude of each (row, warp) cell, top 16 bits rounded up (15 bits for
+            // finite values), and above it the flag "not settled here"
+            const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
+            unsigned int entry = (m0 + 0xffffu) >> 16;
+            if (!COUNTING) {
+                if (PRED) entry |= kFlagBit;
+            } else if (entry > ptl0) {
+                // the cell can reach the lowest band: per candidate the elements above the band's
+                // upper edge, and over all candidates those above the lower edges; the two sums
+                // differ exactly when an element lies inside a band
+                const float a0 = fabsf(u0.x), a1 = fabsf(u0.y), a2 = fabsf(u0.z), a3 = fabsf(u0.w);
+                float h[kUpper];
+#pragma unroll
+                for (int j = 0; j < kUpper; ++j) h[j] = 0.f;
+                float below = 0.f;
+                auto band = [&](const int j) {
+                    const float lo = sh.plo[j], hi = sh.phi[j];
+                    h[j] = (gt_as_float(a0, hi) + gt_as_float(a1, hi)) + (gt_as_float(a2, hi) + gt_as_float(a3, hi));
+                    below += (gt_as_float(a0, lo) + gt_as_float(a1, lo)) + (gt_as_float(a2, lo) + gt_as_float(a3, lo));
+                };
+                band(0);
+                if (entry > ptl1) {
+                    band(1); band(2);
+                    if (entry > ptl3) { band(3); band(4); band(5); }
+                }
+                const float above = ((h[0] + h[1]) + (h[2] + h[3])) + (h[4] + h[5]);
+                if (__any_sync(0xffffffffu, below != above)) {
+                    entry |= kFlagBit;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kUpper / 2; ++j) pacc[j] += fmaf(h[2 * j + 1], kPackScale, h[2 * j]);
+                }
+            }
+            if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)entry;
+        };
+
+        // The rows stream in three stretches: the first kStages - 1 rows, behind whose copies the
+        // sample's were issued; then, the sample having landed, every warp hands its sums in
+        // (between the loops: a call inside a streaming loop would cost registers in every
+        // iteration) and the rows go on until the predicted bands are there; from then on with
+        // the counting.  Each warp changes over by itself, at a row of its own: a cell is
+        // flagged or settled by the one warp that handles it.  Warp 0 reads the band block once
+        // per row (the load is issued before the row and looked at after it) and gives up after
+        // a third of its rows.
+        int r = 0;
+        int64_t i = first4;
+        if (nrows > 0) { row_body(0, i, std::false_type{}); r = 1; i += stride4; }
+        if (PRED) {
+            gring[(size_t)kStages * kRowF4 + tid] = sample_g;
+            if (ACC) gring[(size_t)(kStages + 1) * kRowF4 + tid] = sample_e;
+        }
+        for (; r < nrows && r < kStages - 1; ++r, i += stride4) row_body(r, i, std::false_type{});
+        if (PRED) {
+            publish_sample<ACC>(gring, pv, &sh, bars);
+            for (; r < nrows; ++r, i += stride4) {
+                if (r >= kStages) {
+                    const int word = *reinterpret_cast<volatile int*>(&sh.pred_ready);
+                    if (word == 1) break;              // on to the counting stretch
+                    if (word != 0) pred_state = 0;     // no prediction: nothing to wait for
+                }
+                const bool looking = pred_state != 0 && w == 0;
+                if (looking && lane < 5)
+                    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(sums + lane));
+                row_body(r, i, std::false_type{});
+                if (looking) {
+                    const unsigned int in = (unsigned int)__shfl_sync(0xffffffffu, seen, 4);
+                    const bool late = 3 * r >= nrows;   // too late to be worth having
+                    if (in >= (unsigned)G || late) {
+                        const double a1 = __longlong_as_double(__shfl_sync(0xffffffffu, seen, 0)),
+                                     a2 = __longlong_as_double(__shfl_sync(0xffffffffu, seen, 1)),
+                                     a3 = __longlong_as_double(__shfl_sync(0xffffffffu, seen, 2)),
+                                     a4 = __longlong_as_double(__shfl_sync(0xffffffffu, seen, 3));
+                        if (lane == 0) {
+                            const bool ok = in >= (unsigned)G &&
+                                            predict_bands(a1, a2, a3, a4, (double)G * kSampleElems, pv, z, sh.plo, sh.phi);
+                            __threadfence_block();
+                            *reinterpret_cast<volatile int*>(&sh.pred_ready) = ok ? 1 : 2;
+                        }
+                        pred_state = 0;
+                    }
+                }
+            }
+            if (r < nrows) {
+                // top 16 bits of each tier's lowest band edge, rounded down (the edges are positive)
+                ptl0 = __float_as_uint(sh.plo[0]) >> 16;
+                ptl1 = __float_as_uint(sh.plo[1]) >> 16;
+                ptl3 = __float_as_uint(sh.plo[3]) >> 16;
+                for (; r < nrows; ++r, i += stride4) row_body(r, i, std::true_type{});
+            }
+            if (w == 0 && lane == 0 && *reinterpret_cast<volatile int*>(&sh.pred_ready) == 0)
+                *reinterpret_cast<volatile int*>(&sh.pred_ready) = 2;   // nobody waits for bands any more
+        } else {
+            for (; r < nrows; ++r, i += stride4) row_body(r, i, std::false_type{});
+        }
+        cp_async_wait<0>();
+        if (owns_tail) {
+            tail_u = ACC ? src[tail_i] + eps[tail_i] : src[tail_i];
+            if (ACC) eps[tail_i] = tail_u;
+            const double x = (double)tail_u - pv;
+            s0 += x; q0 = fma(x, x, q0);
+        }
+        const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
+        if (tid == 0) partials[c] = part;
+        stamp(1);
+        if (!grid_barrier(&bars[kBarStats], bar_target, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        stamp(2);
+        // every CTA forms the same totals: thread t takes partial t, t + T, ...
+        double s = 0.0, q = 0.0;
+        for (int t = tid; t < G; t += kFusedThreads) {
+            const double2 p = __ldcg(&partials[t]);
+            s += p.x; q += p.y;
+        }
+        const double2 tot = block_sum2<kFusedThreads>(s, q, sh.red);
+        if (tid == 0) {
+            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
+            alg1_thresholds(st, tot.x, tot.y, pv, d, k, z);
+            // candidate indices in ascending order of threshold
+            const bool neg = sh.stats.thres0 < 0.0;
+#pragma unroll
+            for (int j = 0; j < kNumCand; ++j) sh.order[j] = cand_ascending(j, neg);
+            // phase A's counts stand if every exact candidate lies within its predicted band
+            bool fast = PRED && sh.pred_ready == 1 && sh.stats.thres0 > 0.0;
+            if (fast) {
+#pragma unroll
+                for (int j = 0; j < kUpper; ++j) {
+                    const float cj = sh.cand32[cand_by_factor(kNumCand - kUpper + j)];
+                    fast = fast && sh.plo[j] <= cj && cj <= sh.phi[j];
+                }
+            }
+            sh.fast = fast ? 1 : 0;
+            if (PRED && sh.pred_ready == 1) atomicAdd(&bars[kBarInfo + 0], 1u);
+            sh.recount = 0;
+        }
+        if (tid < kNumCand) sh.cta_counts[tid] = 0u;
+        if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
+        __syncthreads();
+    }
+
+    // ------------------------------------------------------------------ phase B and the rounds
+    // First count: the short way where this CTA's prediction held, else in full.  If the rounds
+    // then ask for a candidate that some CTA left out, the CTAs that took the short way count
+    // again in full and the sums are formed a second time.
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool fast = PRED && pass == 0 && sh.fast != 0;
+        if (fast) count_short_way(uvec, d, n_rows, u_slots, pacc[0], pacc[1], pacc[2], tail_u, bars);
+        else if (pass == 0 || sh.fast != 0) count_in_full(uvec, d, n_rows, u_slots, tail_u, pass == 1);
+        // this CTA's counts join the global sums; the short way leaves the four lower candidates out
+        if (tid < kNumCand) {
+            const unsigned int v = sh.cta_counts[tid];
+            if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
+        }
+        if (fast && tid == 0) {
+            atomicOr(&bars[kBarInvalid], kLowCandMask);
+            atomicAdd(&bars[kBarInfo + 1], 1u);
+        }
+        if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
+        stamp(3);
+        if (!grid_barrier(&bars[pass == 0 ? kBarCounts : kBarCounts2], bar_target, &sh.ok)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+        if (c == 0 && tid == 0) ctrl->phase_t[3] = global_timer_ns();
+        stamp(4);
+
+        // -------------------------------------------------------------- the rounds
+        if (tid < kNumCand) sh.col[tid] = (unsigned long long)ld_acquire_u32((pass == 0 ? tot0 : tot1) + tid);
+        __syncthreads();
+        if (tid == 0) {
+            const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
+            unsigned int visited = 0u;
+            sh.chosen = alg1_resolve(st, k, &visited);
+            sh.n_staged = 0u;
+            // a candidate the rounds evaluated but some CTA did not count: count again, in full
+            sh.recount = (pass == 0 && (visited & ld_acquire_u32(&bars[kBarInvalid])) != 0u) ? 1 : 0;
+        }
+        __syncthreads();
+        if (!sh.recount) break;
+        if (c == 0 && tid == 0) bars[kBarInfo + 2] = 1u;
+    }
+    if (c == 0 && tid == 0) {
+        const long long all = sh.stats.nnz;
+        const long long written = all < cap ? all : cap;
+        // every field but the status word, which was cleared at the start and only ever has
+        // flags added to it (a CTA that gave up waiting may have added one already)
+        gk_stats* o = &ctrl->stats;
+        o->mu = sh.stats.mu; o->sigma = sh.stats.sigma; o->z = sh.stats.z;
+        o->thres0 = sh.stats.thres0; o->thr_final = sh.stats.thr_final;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o->counts[j] = sh.stats.counts[j];
+        o->rounds = sh.stats.rounds; o->nnz = all; o->emitted = written;
+        const int flags = sh.stats.status | (all > cap ? GK_DEV_TRUNCATED : 0);
+        if (flags) atomicOr(&o->status, flags);
+        *nnz_out = written;
+        ctrl->phase_t[4] = global_timer_ns();
+    }
+
+    // ------------------------------------------------------------------ phase C
+    // The survivor count of the whole vector is known to every CTA; with none there is nothing
+    // left to do (the same decision in every CTA, so the barrier inside is reached by all or none).
+    if (sh.stats.nnz != 0) {
+        if (!compact_survivors<ACC>(uvec, eps, d, n_rows, u_slots, bar_target, bars, rowcnt, idx_out, val_out, cap,
+                                    tail_u, trace)) {
+            if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
+            goto leave;
+        }
+    }
+
     if (c == 0 && tid == 0) ctrl->phase_t[5] = global_timer_ns();
     stamp(7);
 
@@ -875,9 +1104,10 @@ leave:
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[6] = global_timer_ns();
             bars[kBarStats] = 0u; bars[kBarCounts] = 0u; bars[kBarRows] = 0u;
-            bars[kBarPublished] = 0u; bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
+            bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
             for (int j = 0; j < 2 * kNumCand; ++j) bars[kBarTotals + j] = 0u;
             for (int j = 0; j < 4; ++j) { ctrl->path_info[j] = bars[kBarInfo + j]; bars[kBarInfo + j] = 0u; }
+            for (int j = 0; j < 9; ++j) bars[kBarSample + j] = 0u;
             __threadfence();
             bars[kBarExit] = 0u;
         }
@@ -891,15 +1121,15 @@ struct FusedPlan {
 };
 static FusedPlan g_plan[64];
 
-template <bool ACC>
+template <bool ACC, bool PRED>
 static bool fused_kernel_ready() {
-    if (cudaFuncSetAttribute(k_gk_fused<ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBudget) !=
+    if (cudaFuncSetAttribute(k_gk_fused<ACC, PRED>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBudget + kFusedStaticBytes) !=
         cudaSuccess) {
         cudaGetLastError();
         return false;
     }
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused<ACC>, kFusedThreads, kFusedSmemBudget) !=
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_gk_fused<ACC, PRED>, kFusedThreads, kFusedSmemBudget + kFusedStaticBytes) !=
             cudaSuccess || occ < 1) {
         cudaGetLastError();
         return false;
@@ -917,7 +1147,8 @@ static FusedPlan* fused_plan(int dev, int sm_count) {
     p.ready = true;
     int coop = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return &p;
-    if (!fused_kernel_ready<true>() || !fused_kernel_ready<false>()) return &p;
+    if (!fused_kernel_ready<true, false>() || !fused_kernel_ready<false, false>() ||
+        !fused_kernel_ready<true, true>() || !fused_kernel_ready<false, true>()) return &p;
     p.grid = sm_count < kFusedMaxGrid ? sm_count : kFusedMaxGrid;
     p.usable = true;
     return &p;
@@ -950,38 +1181,40 @@ static FusedGeometry fused_geometry(int64_t d, int grid) {
     // (with fewer slots than rows in flight the kernel takes eps through the ring instead; the
     // last row of the vector, which may be short, must stay on chip: one slot at least)
     if (q.u_slots < 1) q.fits = false;
-    q.smem = (size_t)(kRing + q.u_slots) * kRowBytes + (size_t)q.table_rows * kTableRowBytes;
+    q.smem = (size_t)kFusedStaticBytes + (size_t)(kRing + q.u_slots) * kRowBytes + (size_t)q.table_rows * kTableRowBytes;
     return q;
 }
 
 // Whether the call counts during phase A against predicted thresholds: on vectors large enough
 // for the prediction to arrive early in a CTA's run (a test hook can force either answer).
-static int wants_prediction(const FusedGeometry& geo, int64_t d) {
-    const bool possible = (d >> 7) >= 1;   // one block of 32 float4 at least
+static bool wants_prediction(const FusedGeometry& geo, int64_t d) {
+    // one block of 32 float4 at least; a thread's packed counts hold kPredMaxRows rows
+    // (and eps arriving in the u slots, which leaves the ring's upper half to the sample)
+    const bool possible = (d >> 7) >= 1 && geo.table_rows <= kPredMaxRows && geo.u_slots >= kStages;
     const int knob = host_knob(kKnobPrediction);
-    if (knob == 0 || !possible) return 0;
-    if (knob == 1) return 1;
-    return (int64_t)geo.n_rows >= (int64_t)kPredMinRows * geo.G ? 1 : 0;
+    if (knob == 0 || !possible) return false;
+    if (knob == 1) return true;
+    return (int64_t)geo.n_rows >= (int64_t)kPredMinRows * geo.G;
 }
 
 // The one place that builds the kernel's argument list (types checked by the compiler).
 // eps == nullptr launches the operator form.
 static cudaError_t launch_fused(const FusedGeometry& geo, cudaStream_t st, const float* src, float* eps, int64_t d,
-                                int64_t k, double z, Ctrl* ctrl, double2* partials, double2* spart,
-                                unsigned int* bars, unsigned int* rowcnt, int32_t* idx_out, float* val_out,
+                                int64_t k, double z, Ctrl* ctrl, double2* partials, unsigned int* bars, unsigned int* rowcnt, int32_t* idx_out, float* val_out,
                                 int64_t* nnz_out, int64_t cap, unsigned long long* trace) {
     int n_rows = geo.n_rows, u_slots = geo.u_slots, table_rows = geo.table_rows;
-    int predict = wants_prediction(geo, d);
     unsigned int bar_target = (unsigned int)geo.G + (unsigned int)host_knob(kKnobExtraArrivals);
     void* args[] = {(void*)&src, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&n_rows, (void*)&u_slots,
-                    (void*)&table_rows, (void*)&predict, (void*)&bar_target, (void*)&ctrl, (void*)&partials,
-                    (void*)&spart, (void*)&bars, (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out,
-                    (void*)&cap, (void*)&trace};
-    static_assert(sizeof(args) / sizeof(args[0]) == 20, "k_gk_fused takes 20 arguments");
-    // the two instances have the same parameter list; naming them keeps the types checked
-    void (*kern)(const float*, float*, int64_t, int64_t, double, int, int, int, int, unsigned int, Ctrl*, double2*,
-                 double2*, unsigned int*, unsigned int*, int32_t*, float*, int64_t*, int64_t, unsigned long long*) =
-        eps != nullptr ? k_gk_fused<true> : k_gk_fused<false>;
+                    (void*)&table_rows, (void*)&bar_target, (void*)&ctrl, (void*)&partials,
+                    (void*)&bars, (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap,
+                    (void*)&trace};
+    static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused takes 18 arguments");
+    // the four instances have the same parameter list; naming them keeps the types checked
+    typedef void (*Kern)(const float*, float*, int64_t, int64_t, double, int, int, int, unsigned int, Ctrl*, double2*,
+                         unsigned int*, unsigned int*, int32_t*, float*, int64_t*, int64_t, unsigned long long*);
+    const bool acc = eps != nullptr, pred = wants_prediction(geo, d);
+    const Kern kern = acc ? (pred ? (Kern)k_gk_fused<true, true> : (Kern)k_gk_fused<true, false>)
+                          : (pred ? (Kern)k_gk_fused<false, true> : (Kern)k_gk_fused<false, false>);
     return cudaLaunchCooperativeKernel((const void*)kern, dim3((unsigned)geo.G), dim3(kFusedThreads), args,
                                        geo.smem, st);
 }
@@ -1001,9 +1234,7 @@ int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int
     const double z = normal_quantile_upper(1.0 - pq);
     ws->last_grid = (int)geo.G;
     stage_mark(ws, st, 0);
-    // the sample sums sit behind the per-CTA partials (at most kFusedGridCap of them)
-    GK_CUDA_TRY(launch_fused(geo, st, src, eps, d, k, z, ws->ctrl, ws->partials, ws->partials + kFusedGridCap, ws->bars,
-                             ws->rowcnt, idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
+    GK_CUDA_TRY(launch_fused(geo, st, src, eps, d, k, z, ws->ctrl, ws->partials, ws->bars, ws->rowcnt, idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_fused = true;
@@ -1030,7 +1261,7 @@ int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int
 namespace gk {
 
 constexpr size_t kStaticCtrlBytes = (sizeof(Ctrl) + 255) / 256 * 256;
-constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap * 3;   // 24 KB: partial sums, then sample sums
+constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap;                // 8 KB
 constexpr size_t kStaticBarBytes = sizeof(unsigned int) * kBarWords;          // 256 bytes
 constexpr size_t kStaticHeadBytes = 32 * 1024;             // everything but the per-row words
 constexpr int kStaticRowCap = 1 << 17;                     // rows of 4096 elements: d up to 2^29
@@ -1096,8 +1327,8 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
     const double pq = 1.0 - (double)k / (double)d;
     const double z = normal_quantile_upper(1.0 - pq);
     unsigned long long* trace = nullptr;  // no trace array in the fixed scratch
-    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, partials + kFusedGridCap, bars, rowcnt, idx_out,
-                             val_out, nnz_out, output_capacity(d), trace));
+    GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, bars, rowcnt, idx_out, val_out, nnz_out,
+                             output_capacity(d), trace));
     note_launch();
     return GK_OK;
 }
