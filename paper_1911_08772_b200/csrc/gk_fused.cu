@@ -93,6 +93,7 @@ constexpr int kSampleElems = kFusedThreads * 4;   // sample elements per CTA: on
 constexpr double kPredSigmas = 3.5;     // half width of the bands in standard errors of the predicted threshold
 constexpr double kPredSlack = 5e-4;     // added to the relative half width
 constexpr double kPredMaxDelta = 0.05;  // wider bands than this are not worth counting against
+constexpr unsigned int kSparseWay = 2;  // no prediction: the short way is taken when at most 1 cell in 2 is loud
 constexpr unsigned int kFlagBit = 0x8000u;   // table entry: the cell was not settled in phase A
 constexpr unsigned int kMaxMask = 0x7fffu;   // table entry: the cell's maximum (top 16 bits, rounded up)
 // candidates that only phase B's full count covers
@@ -350,34 +351,60 @@ __device__ __forceinline__ Smem smem_of(const int u_slots) {
     (void)gring; (void)uslot; (void)table; (void)lane; (void)w; (void)c; (void)G; (void)nrows; (void)first_kept; \
     (void)n4; (void)stride4; (void)first4; (void)tail_i; (void)in_last_row; (void)owns_tail; (void)sh
 
+// Without a prediction every cell is still to be counted after phase A.  Where few of this
+// CTA's cells can reach even thres0 / 2 (loud layers among quiet ones, heavy tails), the short
+// way over those few -- the six upper candidates and thres0 / 2, which the rounds visit when
+// the first count falls short -- beats streaming every row again; the three lowest candidates
+// then wait for the rounds to ask for them.  Sets sh.fast.  Out of line.
+__device__ __noinline__ void decide_sparse_way(const int64_t d, const int n_rows, const int u_slots) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
+    if (tid == 0) sh.samp_n = 0u;
+    __syncthreads();
+    const unsigned int lim = __float_as_uint(fmaxf(sh.cand32[cand_by_factor(kNumCand - kUpper - 1)], 0.f)) >> 16;
+    unsigned int loud = 0u;
+    for (int rr = lane; rr < nrows; rr += 32) loud += (((unsigned int)table[rr * kFusedWarps + w] & kMaxMask) > lim) ? 1u : 0u;
+    loud = __reduce_add_sync(0xffffffffu, loud);
+    if (lane == 0 && loud) atomicAdd(&sh.samp_n, loud);
+    __syncthreads();
+    if (tid == 0) sh.fast = (sh.stats.thres0 > 0.0 && sh.samp_n * kSparseWay <= (unsigned int)nrows * kFusedWarps) ? 1 : 0;
+}
+
 // Phase B, the short way: the six upper candidates over the cells that phase A left (flagged),
 // added to phase A's own counts (pacc, two candidates to a float).  The cells are few and
 // scattered, so every warp gathers its own eight at a time and loads them together, from shared
 // memory where the row is on chip, else from L2.  Leaves the CTA's counts in sh.cta_counts.
 // Out of line: its registers are its own.
+template <int NC>
 __device__ __noinline__ void count_short_way(const float* __restrict__ uvec, const int64_t d, const int n_rows,
                                              const int u_slots, const float pacc0, const float pacc1,
                                              const float pacc2, const float tail_u, unsigned int* __restrict__ bars) {
+    static_assert(NC == kUpper || NC == kUpper + 1, "the six upper candidates, or those and thres0 / 2");
     GK_FUSED_VIEW(d, n_rows, u_slots);
     const float4* u4 = reinterpret_cast<const float4*>(uvec);
     const float pacc[kUpper / 2] = {pacc0, pacc1, pacc2};
-    float cs[kUpper], acc[kUpper];
+    constexpr int X = NC - kUpper;   // candidates below the six upper ones
+    float cs[NC], acc[NC];
 #pragma unroll
-    for (int j = 0; j < kUpper; ++j) cs[j] = sh.cand32[cand_by_factor(kNumCand - kUpper + j)];
+    for (int j = 0; j < NC; ++j) { cs[j] = sh.cand32[cand_by_factor(kNumCand - NC + j)]; acc[j] = 0.f; }
 #pragma unroll
     for (int j = 0; j < kUpper / 2; ++j) {
         const float hi = floorf(pacc[j] * (1.0f / kPackScale));
-        acc[2 * j] = pacc[j] - hi * kPackScale;
-        acc[2 * j + 1] = hi;
+        acc[X + 2 * j] = pacc[j] - hi * kPackScale;
+        acc[X + 2 * j + 1] = hi;
     }
-    const unsigned int t0 = __float_as_uint(cs[0]) >> 16, t1 = __float_as_uint(cs[1]) >> 16,
-                       t3 = __float_as_uint(cs[3]) >> 16;
+    // tiers: [thres0 / 2], 3/4, {1, 9/8}, {3/2, 9/4, 27/8}: evaluated as far as the cell's maximum reaches
+    const unsigned int t0 = __float_as_uint(cs[0]) >> 16, tq = __float_as_uint(cs[X]) >> 16,
+                       t1 = __float_as_uint(cs[X + 1]) >> 16, t3 = __float_as_uint(cs[X + 3]) >> 16;
     auto count_upper = [&](const float4 x, const unsigned int rm) {   // rm > t0
         const float a0 = fabsf(x.x), a1 = fabsf(x.y), a2 = fabsf(x.z), a3 = fabsf(x.w);
-        count_tier<0, 1>(a0, a1, a2, a3, cs, acc);
+        if (X == 1) {
+            count_tier<0, 1>(a0, a1, a2, a3, cs, acc);
+            if (rm <= tq) return;
+        }
+        count_tier<X, X + 1>(a0, a1, a2, a3, cs, acc);
         if (rm > t1) {
-            count_tier<1, 3>(a0, a1, a2, a3, cs, acc);
-            if (rm > t3) count_tier<3, kUpper>(a0, a1, a2, a3, cs, acc);
+            count_tier<X + 1, X + 3>(a0, a1, a2, a3, cs, acc);
+            if (rm > t3) count_tier<X + 3, NC>(a0, a1, a2, a3, cs, acc);
         }
     };
     unsigned int n_left = 0u;   // cells this warp had left
@@ -396,21 +423,19 @@ __device__ __noinline__ void count_short_way(const float* __restrict__ uvec, con
         }
 #pragma unroll
         for (int q = 0; q < kGroupRows; ++q) {
-            if (q < n) {
-                count_upper(v[q], (unsigned int)table[sh.qrow[w][q] * kFusedWarps + w] & kMaxMask);
-            }
+            if (q < n) count_upper(v[q], (unsigned int)table[sh.qrow[w][q] * kFusedWarps + w] & kMaxMask);
         }
         __syncwarp();
     }
     if (owns_tail) {
         const float a = fabsf(tail_u);
 #pragma unroll
-        for (int j = 0; j < kUpper; ++j) acc[j] += gt_as_float(a, cs[j]);
+        for (int j = 0; j < NC; ++j) acc[j] += gt_as_float(a, cs[j]);
     }
 #pragma unroll
-    for (int j = 0; j < kUpper; ++j) {
+    for (int j = 0; j < NC; ++j) {
         const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
-        if (lane == 0 && ws) atomicAdd(&sh.cta_counts[cand_by_factor(kNumCand - kUpper + j)], ws);
+        if (lane == 0 && ws) atomicAdd(&sh.cta_counts[cand_by_factor(kNumCand - NC + j)], ws);
     }
     if (lane == 0 && n_left) atomicAdd(&bars[kBarInfo + 3], n_left);
     __syncthreads();
@@ -887,7 +912,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             const unsigned int m0 = __reduce_max_sync(0xffffffffu, one ? max_mag_bits(u0) : 0u);
             unsigned int entry = (m0 + 0xffffu) >> 16;
             if (!COUNTING) {
-                if (PRED) entry |= kFlagBit;
+                entry |= kFlagBit;
             } else if (entry > ptl0) {
                 // the cell can reach the lowest band: per candidate the elements above the band's
                 // upper edge, and over all candidates those above the lower edges; the two sums
@@ -1019,6 +1044,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             sh.recount = 0;
         }
         if (tid < kNumCand) sh.cta_counts[tid] = 0u;
+        if (!PRED) decide_sparse_way(d, n_rows, u_slots);
         if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
         __syncthreads();
     }
@@ -1028,8 +1054,11 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
     // then ask for a candidate that some CTA left out, the CTAs that took the short way count
     // again in full and the sums are formed a second time.
     for (int pass = 0; pass < 2; ++pass) {
-        const bool fast = PRED && pass == 0 && sh.fast != 0;
-        if (fast) count_short_way(uvec, d, n_rows, u_slots, pacc[0], pacc[1], pacc[2], tail_u, bars);
+        const bool fast = pass == 0 && sh.fast != 0;
+        if (fast) {
+            if (PRED) count_short_way<kUpper>(uvec, d, n_rows, u_slots, pacc[0], pacc[1], pacc[2], tail_u, bars);
+            else count_short_way<kUpper + 1>(uvec, d, n_rows, u_slots, 0.f, 0.f, 0.f, tail_u, bars);
+        }
         else if (pass == 0 || sh.fast != 0) count_in_full(uvec, d, n_rows, u_slots, tail_u, pass == 1);
         // this CTA's counts join the global sums; the short way leaves the four lower candidates out
         if (tid < kNumCand) {
@@ -1037,7 +1066,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
         }
         if (fast && tid == 0) {
-            atomicOr(&bars[kBarInvalid], kLowCandMask);
+            atomicOr(&bars[kBarInvalid], PRED ? kLowCandMask : (kLowCandMask & ~(1u << cand_index(1, 0))));
             atomicAdd(&bars[kBarInfo + 1], 1u);
         }
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
