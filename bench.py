@@ -335,7 +335,10 @@ def run_ours(args):
     with sampler:
         first = max_over_ranks(time_region(torch, lambda t: step(W + t), K), world, dev)
         regions.append(first)
-        repeats = 1 if args.loop_only else max(1, min(2000, int(MIN_TIMED_MS / max(first, 1e-3)) + 1))
+        if args.repeats > 0:
+            repeats = args.repeats
+        else:
+            repeats = 1 if args.loop_only else max(1, min(2000, int(MIN_TIMED_MS / max(first, 1e-3)) + 1))
         for rep in range(1, repeats):
             barrier()
             regions.append(max_over_ranks(time_region(torch, lambda t: step(W + rep * K + t), K), world, dev))
@@ -761,6 +764,8 @@ def main():
                     help="0: fused cooperative kernel, 1: three kernels with look-back")
     ap.add_argument("--rotate", type=int, default=0,
                     help="number of gradient buffers kept on the device (default 20; small for captures)")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="times the timed K-step region is run (0: until about 0.3 s have been timed)")
     ap.add_argument("--loop-only", action="store_true",
                     help="run only warm-up and the timed loop (for profiler captures)")
     ap.add_argument("--call", default="gk", choices=["gk", "gk_select", "segmented", "topk_exact", "topk_sparsify", "dgck_select", "dgck_sparsify"],

@@ -296,6 +296,19 @@ int gk_histogram(const float* u, int64_t d, float lo, float inv_w, int32_t nbins
 int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                        float* val_out, int64_t* nnz_out, gk_stream_t stream);
 
+/*
+ * gk_set_params -- the two constants of Algorithm 1 that can be read in more than one way.
+ *   unbiased_std  non-zero (default): "std" is the sample standard deviation, divisor d - 1
+ *                 (the paper's operators are tensor-library calls whose default this is);
+ *                 0: the population form, divisor d.
+ *   max_rounds    rounds of the loop "for i = 0 -> 3": 4 by default (both bounds included),
+ *                 1 .. 4 accepted; the mask of the last round run is returned.
+ * Applies to gk_sparsify, gk_select, gk_sparsify_segmented, gk_sparsify_host and
+ * gk_sparsify_static from the next call on.  Process-wide; the device-side values are set on
+ * the current device.  Returns GK_ERR_SIZE for max_rounds outside 1 .. 4.
+ */
+int gk_set_params(int unbiased_std, int max_rounds);
+
 /* Output capacity of idx_out / val_out for the sparsify calls, in pairs.
  * 0 (the default) means "d".  Process-wide; returns GK_ERR_CAPACITY if cap < 0. */
 int gk_set_capacity(int64_t cap);

@@ -26,7 +26,7 @@ EXPORTS = [
     "gk_sparsify_static", "gk_set_capacity", "gk_set_path", "gk_reserve", "gk_workspace_bytes", "gk_last_stats", "gk_last_segment_stats",
     "gk_stage_timing", "gk_last_stage_ms", "gk_last_cta_trace", "gk_launch_count", "gk_strerror", "gk_last_cuda_error", "gk_version",
     "gk_error_ratio", "dgck_select", "dgck_sparsify", "dgck_last_info",
-    "gk_apply_sparse", "gk_apply_gathered", "gk_histogram", "gk_debug_set", "gk_last_path_info", "gk_select",
+    "gk_apply_sparse", "gk_apply_gathered", "gk_histogram", "gk_debug_set", "gk_last_path_info", "gk_select", "gk_set_params",
 ]
 
 
@@ -119,6 +119,8 @@ def load() -> C.CDLL:
     L.gk_version.argtypes = []
     L.gk_last_path_info.argtypes = [vp, C.POINTER(i64)]
     L.gk_last_path_info.restype = C.c_int
+    L.gk_set_params.argtypes = [C.c_int, C.c_int]
+    L.gk_set_params.restype = C.c_int
     L.gk_debug_set.argtypes = [C.c_int, i64]
     L.gk_debug_set.restype = C.c_int
     for name in ("gk_sparsify", "gk_sparsify_segmented", "topk_exact", "topk_sparsify", "gk_sparsify_host",
@@ -278,6 +280,11 @@ def gk_sparsify_host(g, eps, k: int, idx_out, val_out):
 
 def gk_set_capacity(cap: int) -> None:
     _check(load().gk_set_capacity(cap))
+
+
+def gk_set_params(unbiased_std: bool = True, max_rounds: int = 4) -> None:
+    """Divisor of the variance (d - 1 or d) and number of rounds of Algorithm 1 (see gk.h)."""
+    _check(load().gk_set_params(int(bool(unbiased_std)), max_rounds))
 
 
 def gk_set_path(path: int) -> None:

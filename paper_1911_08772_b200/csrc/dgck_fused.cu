@@ -238,24 +238,8 @@ k_dgck_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
         __syncthreads();
 
         auto gather = [&](int& cursor, const bool want_pending) -> int {
-            int nq = 0;
-            while (nq < kTkGroupRows && cursor < nrows) {
-                const int r = cursor + lane;
-                unsigned int e = 0u;
-                if (r < nrows) e = table[r * kFusedWarps + w];
-                const bool hit = want_pending ? (e == kTkPending) : (e != 0u);
-                unsigned int b = __ballot_sync(0xffffffffu, hit);
-                while (b && nq < kTkGroupRows) {
-                    const int bit = __ffs(b) - 1;
-                    if (lane == 0) sh.qrow[w][nq] = (unsigned short)(cursor + bit);
-                    ++nq;
-                    b &= b - 1u;
-                }
-                if (b) { cursor += __ffs(b) - 1; break; }
-                cursor += 32;
-            }
-            __syncwarp();
-            return nq;
+            return want_pending ? gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w])
+                                : gather_cells<kGatherNonZero>(table, nrows, cursor, sh.qrow[w]);
         };
         auto load_row = [&](int r) -> float4 {
             const int64_t i = first4 + (int64_t)r * stride4;

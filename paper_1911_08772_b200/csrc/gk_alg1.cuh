@@ -49,6 +49,20 @@ __host__ __device__ constexpr int cand_ascending(int j, bool thres0_negative) {
     return cand_by_factor(thres0_negative ? kNumCand - 1 - j : j);
 }
 
+#ifdef __CUDACC__
+// The two constants of Algorithm 1 that the paper leaves open to reading (gk_set_params): the
+// divisor of the variance (d - 1 by default, d when `biased`) and the number of rounds (4 by
+// default).  One copy per translation unit, set through the registered setter.
+static __device__ int g_alg1_biased = 0;
+static __device__ int g_alg1_max_rounds = kMaxRounds;
+static int set_alg1_knob(int key, int value) {
+    if (key == kKnobBiasedStd) return (int)cudaMemcpyToSymbol(g_alg1_biased, &value, sizeof(int));
+    if (key == kKnobMaxRounds) return (int)cudaMemcpyToSymbol(g_alg1_max_rounds, &value, sizeof(int));
+    return 0;
+}
+static const int g_alg1_knob_registered = register_knob_setter(&set_alg1_knob);
+#endif
+
 // Where one run of Algorithm 1 keeps its scalars.
 struct Alg1State {
     gk_stats* stats;
@@ -80,7 +94,7 @@ __device__ inline void alg1_thresholds(const Alg1State& a, double s1, double s2,
     }
     const double dn = (double)n;
     const double mean_shift = s1 / dn;
-    double var = (s2 - s1 * mean_shift) / (dn - 1.0);  // sample variance
+    double var = (s2 - s1 * mean_shift) / (g_alg1_biased ? dn : dn - 1.0);  // sample variance unless asked otherwise
     if (var < 0.0) var = 0.0;
     st.mu = c + mean_shift;
     st.sigma = sqrt(var);
@@ -119,12 +133,13 @@ __device__ inline Alg1Path alg1_replay(const unsigned long long* counts, int64_t
     p.visited = 0u;
     int h = 0, b = 0;
     bool going = true;
+    const int max_rounds = g_alg1_max_rounds;
     // four rounds at most, written out so that nothing is indexed by a run-time value (arrays
     // indexed that way live in local memory, and one thread walks this chain for the whole grid)
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
         long long est = 0;
-        if (going) {
+        if (going && r < max_rounds) {
             const int ci = cand_index(h, b);
             // the counts may live in global or in shared memory: a generic volatile load serves both
             est = (long long)*reinterpret_cast<const volatile unsigned long long*>(&counts[ci]);

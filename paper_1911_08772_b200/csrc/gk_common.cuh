@@ -42,7 +42,9 @@ enum Knob {
     kKnobExtraArrivals = 2,   // host: arrivals the fused kernels' barriers expect beyond the grid size
     kKnobMuteTile = 3,        // compaction tile that does not publish its status word (-1: none)
     kKnobPrediction = 4,      // host: -1 automatic, 0 never, 1 whenever possible (gk_fused.cu)
-    kKnobCount = 5
+    kKnobBiasedStd = 5,       // gk_set_params: 1 divides the variance by d instead of d - 1
+    kKnobMaxRounds = 6,       // gk_set_params: rounds of Algorithm 1's loop, 1 .. 4
+    kKnobCount = 7
 };
 typedef int (*KnobSetter)(int key, int value);   // returns a cudaError_t as int
 int register_knob_setter(KnobSetter fn);

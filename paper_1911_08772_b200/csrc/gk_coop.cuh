@@ -62,6 +62,42 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
     return *ok_flag != 0;
 }
 
+// The per-(row, warp) table of the persistent kernels: one uint16 per cell of 128 elements.
+constexpr int kGroupRows = 8;                // rows a warp gathers per batch
+constexpr unsigned int kFlagBit = 0x8000u;   // fused sparsifier: the cell has not been counted yet
+constexpr unsigned int kMaxMask = 0x7fffu;   // fused sparsifier: the cell's maximum (top 16 bits, rounded up)
+
+// Up to kGroupRows of this warp's cells (local rows) that meet a condition, from row `cursor`
+// on: their rows go to qrow[0 ..), the cursor moves past the last one taken.  Called by all
+// lanes of a warp; returns the number of rows gathered.
+enum GatherWhat { kGatherFlagged, kGatherPending, kGatherNonZero };
+constexpr unsigned short kPending = 0xffffu;   // the cell is marked, its count is still to come
+template <GatherWhat WHAT>
+__device__ __forceinline__ int gather_cells(const unsigned short* table, const int nrows, int& cursor,
+                                            unsigned short* qrow, const unsigned int above = 0u) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int n = 0;
+    while (n < kGroupRows && cursor < nrows) {
+        const int r = cursor + lane;
+        unsigned int e = 0u;
+        if (r < nrows) e = table[r * kFusedWarps + w];
+        // (flagged cells only count when their maximum reaches the lowest threshold of interest)
+        const bool hit = WHAT == kGatherFlagged ? (e & kFlagBit) != 0u && (e & kMaxMask) > above
+                         : WHAT == kGatherPending ? e == kPending : e != 0u;
+        unsigned int b = __ballot_sync(0xffffffffu, hit);
+        while (b && n < kGroupRows) {
+            const int bit = __ffs(b) - 1;
+            if (lane == 0) qrow[n] = (unsigned short)(cursor + bit);
+            ++n;
+            b &= b - 1u;
+        }
+        if (b) { cursor += __ffs(b) - 1; break; }
+        cursor += 32;
+    }
+    __syncwarp();
+    return n;
+}
+
 #endif  // __CUDACC__
 
 }  // namespace gk

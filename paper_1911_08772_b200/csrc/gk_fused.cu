@@ -72,7 +72,6 @@ constexpr int kTableRowBytes = kFusedWarps * 2;        // one uint16 per (row, w
 constexpr int kFusedSmemBudget = 221184;               // dynamic shared memory the kernel may ask for
 constexpr int kStages = 4;                             // phase A: rows of g and eps in flight, plus one
 constexpr int kRing = 8;                               // ring slots; phase B has kRing - 1 rows in flight
-constexpr int kGroupRows = 8;                          // rows a warp gathers per batch in phase C
 constexpr int kFusedMaxGrid = kFusedGridCap;
 constexpr int kTraceSlots = 8;                         // timestamps per CTA in the optional trace
 // phase C keeps the places of a CTA's survivors (row, warp, lane, element, rank within the
@@ -94,8 +93,6 @@ constexpr double kPredSigmas = 3.5;     // half width of the bands in standard e
 constexpr double kPredSlack = 5e-4;     // added to the relative half width
 constexpr double kPredMaxDelta = 0.05;  // wider bands than this are not worth counting against
 constexpr unsigned int kSparseWay = 2;  // no prediction: the short way is taken when at most 1 cell in 2 is loud
-constexpr unsigned int kFlagBit = 0x8000u;   // table entry: the cell was not settled in phase A
-constexpr unsigned int kMaxMask = 0x7fffu;   // table entry: the cell's maximum (top 16 bits, rounded up)
 // candidates that only phase B's full count covers
 constexpr unsigned int kLowCandMask = (1u << cand_index(1, 0)) | (1u << cand_index(2, 0)) |
                                       (1u << cand_index(3, 0)) | (1u << cand_index(2, 1));
@@ -190,37 +187,6 @@ __device__ __noinline__ bool predict_bands(double s1, double s2, double s3, doub
         phi[j] = __double2float_ru(th * f[j] * up);
     }
     return phi[kUpper - 1] < 3.0e38f;
-}
-
-// Up to kGroupRows of this warp's cells (local rows) that meet a condition, from row `cursor`
-// on: their rows go to qrow[0 ..), the cursor moves past the last one taken.  Called by all
-// lanes of a warp; returns the number of rows gathered.
-enum GatherWhat { kGatherFlagged, kGatherPending, kGatherNonZero };
-constexpr unsigned short kPending = 0xffffu;   // phase C: the cell qualifies, its count is still to come
-template <GatherWhat WHAT>
-__device__ __forceinline__ int gather_cells(const unsigned short* table, const int nrows, int& cursor,
-                                            unsigned short* qrow, const unsigned int above = 0u) {
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    int n = 0;
-    while (n < kGroupRows && cursor < nrows) {
-        const int r = cursor + lane;
-        unsigned int e = 0u;
-        if (r < nrows) e = table[r * kFusedWarps + w];
-        // (flagged cells only count when their maximum reaches the lowest threshold of interest)
-        const bool hit = WHAT == kGatherFlagged ? (e & kFlagBit) != 0u && (e & kMaxMask) > above
-                         : WHAT == kGatherPending ? e == kPending : e != 0u;
-        unsigned int b = __ballot_sync(0xffffffffu, hit);
-        while (b && n < kGroupRows) {
-            const int bit = __ffs(b) - 1;
-            if (lane == 0) qrow[n] = (unsigned short)(cursor + bit);
-            ++n;
-            b &= b - 1u;
-        }
-        if (b) { cursor += __ffs(b) - 1; break; }
-        cursor += 32;
-    }
-    __syncwarp();
-    return n;
 }
 
 // The sample of one CTA: warp w reads block (c * 32 + w) of G * 32 blocks of 32 float4 spread

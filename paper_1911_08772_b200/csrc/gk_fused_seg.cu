@@ -632,24 +632,8 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             return m;
         };
         auto gather = [&](int& cursor, const bool want_pending) -> int {
-            int n = 0;
-            while (n < kSfGroupRows && cursor < nrows) {
-                const int r = cursor + lane;
-                unsigned int e = 0u;
-                if (r < nrows) e = table[r * kFusedWarps + w];
-                const bool hit = want_pending ? (e == kSfPending) : (e != 0u);
-                unsigned int b = __ballot_sync(0xffffffffu, hit);
-                while (b && n < kSfGroupRows) {
-                    const int bit = __ffs(b) - 1;
-                    if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
-                    ++n;
-                    b &= b - 1u;
-                }
-                if (b) { cursor += __ffs(b) - 1; break; }
-                cursor += 32;
-            }
-            __syncwarp();
-            return n;
+            return want_pending ? gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w])
+                                : gather_cells<kGatherNonZero>(table, nrows, cursor, sh.qrow[w]);
         };
         auto load_row = [&](int r, int64_t i) -> float4 {
             return (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : __ldcg(e4 + i);

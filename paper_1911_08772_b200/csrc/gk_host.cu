@@ -170,17 +170,27 @@ extern "C" int gk_set_path(int path) {
     return GK_OK;
 }
 
-extern "C" int gk_debug_set(int key, int64_t value) {
-    if (key < 0 || key >= kKnobCount || value < -1 || value > 2147483647ll) return GK_ERR_SIZE;
-    g_host_knob[key].store((int)value);
+static int set_knob_everywhere(int key, int value) {
+    g_host_knob[key].store(value);
     g_host_knob_set[key].store(true);
     KnobRegistry& r = knob_registry();
     std::lock_guard<std::mutex> lock(r.mu);
     for (int i = 0; i < r.n; ++i) {
-        const int e = r.fn[i](key, (int)value);
+        const int e = r.fn[i](key, value);
         if (e != 0) return cuda_fail((cudaError_t)e);
     }
     return GK_OK;
+}
+
+extern "C" int gk_set_params(int unbiased_std, int max_rounds) {
+    if (max_rounds < 1 || max_rounds > kMaxRounds) return GK_ERR_SIZE;
+    const int rc = set_knob_everywhere(kKnobBiasedStd, unbiased_std ? 0 : 1);
+    return rc != GK_OK ? rc : set_knob_everywhere(kKnobMaxRounds, max_rounds);
+}
+
+extern "C" int gk_debug_set(int key, int64_t value) {
+    if (key < 0 || key >= kKnobBiasedStd || value < -1 || value > 2147483647ll) return GK_ERR_SIZE;
+    return set_knob_everywhere(key, (int)value);
 }
 
 extern "C" int gk_reserve(int64_t d, int32_t S, gk_stream_t stream) {

@@ -90,24 +90,8 @@ k_topk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, 
     // up to kTkGroupRows rows of this warp whose table entry is pending (want_pending) or
     // non-zero, from `cursor` on; they are left in sh.qrow[w]
     auto gather = [&](int& cursor, const bool want_pending) -> int {
-        int n = 0;
-        while (n < kTkGroupRows && cursor < nrows) {
-            const int r = cursor + lane;
-            unsigned int e = 0u;
-            if (r < nrows) e = table[r * kFusedWarps + w];
-            const bool hit = want_pending ? (e == kTkPending) : (e != 0u);
-            unsigned int b = __ballot_sync(0xffffffffu, hit);
-            while (b && n < kTkGroupRows) {
-                const int bit = __ffs(b) - 1;
-                if (lane == 0) sh.qrow[w][n] = (unsigned short)(cursor + bit);
-                ++n;
-                b &= b - 1u;
-            }
-            if (b) { cursor += __ffs(b) - 1; break; }
-            cursor += 32;
-        }
-        __syncwarp();
-        return n;
+        return want_pending ? gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w])
+                            : gather_cells<kGatherNonZero>(table, nrows, cursor, sh.qrow[w]);
     };
     // this thread's float4 of local row r (zeros beyond the end of the vector)
     auto load_row = [&](int r) -> float4 {

@@ -70,7 +70,8 @@ class DeviceStep:
         return idx[:n].copy(), val[:n].copy(), n
 
 
-def compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, cap, check_counts=True):
+def compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, cap, check_counts=True, max_rounds=4,
+                        unbiased=True):
     """One finished sparsifier step (pairs idx/val[:n], record st, residual eps_new, output
     capacity cap) against the oracle, by the acceptance rule in this module's header.
 
@@ -82,7 +83,7 @@ def compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, cap, check_count
     iteration returns 0 exactly."""
     d = g.shape[0]
     u = orc.accumulate(g, eps_in)
-    ost = orc.gaussiank_threshold(u, k)
+    ost = orc.gaussiank_threshold(u, k, max_rounds=max_rounds, unbiased=unbiased)
     assert st.status in (0, gk.GK_DEV_TRUNCATED)
     if k < d:
         assert rel_close(st.mu, ost.mu, 1e-6) or abs(st.mu - ost.mu) <= 1e-9 * ost.sigma
@@ -107,7 +108,7 @@ def compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, cap, check_count
 
 
 def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, check_counts=True,
-                  call=None):
+                  call=None, max_rounds=4, unbiased=True):
     """Run one gk_sparsify step (or `call`, an entry point with the same arguments) on the
     device and compare with the oracle.  Returns (eps_new (numpy, from the device), stats)."""
     step.g.copy_(torch.from_numpy(g))
@@ -117,7 +118,7 @@ def check_gk_step(step: DeviceStep, g: np.ndarray, eps_in: np.ndarray, k: int, c
     idx, val, n = step.outputs()
     st = gk.gk_last_stats()
     eps_new = step.eps.cpu().numpy()
-    compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, step.cap, check_counts)
+    compare_with_oracle(g, eps_in, k, idx, val, n, st, eps_new, step.cap, check_counts, max_rounds, unbiased)
     return eps_new, st
 
 
