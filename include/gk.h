@@ -314,13 +314,16 @@ int gk_set_params(int unbiased_std, int max_rounds);
 int gk_set_capacity(int64_t cap);
 
 /*
- * Which implementation gk_sparsify (and gk_sparsify_host) uses.  Process-wide.
- *   0 (default)  one persistent cooperative kernel that keeps what fits of u in
- *                shared memory between the phases of Algorithm 1; falls back to
- *                path 1 where cooperative launch is unavailable and for k = d.
+ * Which implementation gk_sparsify, gk_select and gk_sparsify_host use.  Process-wide.
+ *   0 (default)  vectors of up to 589,824 elements: one thread-block cluster of sixteen CTAs
+ *                that holds u in shared memory and synchronises with cluster barriers;
+ *                larger ones: one persistent cooperative kernel that keeps what fits of u in
+ *                shared memory between the phases of Algorithm 1.  Falls back to path 1 where
+ *                neither can be launched and for k = d.
  *   1            three kernels: accumulate + statistics, candidate counts,
  *                compaction by decoupled look-back.
- * Both give identical results.  Returns GK_ERR_SIZE for any other value.
+ *   2            the persistent cooperative kernel at every size.
+ * All give identical results.  Returns GK_ERR_SIZE for any other value.
  */
 int gk_set_path(int path);
 

@@ -288,7 +288,8 @@ def gk_set_params(unbiased_std: bool = True, max_rounds: int = 4) -> None:
 
 
 def gk_set_path(path: int) -> None:
-    """0: fused cooperative kernel (default); 1: three kernels with look-back."""
+    """0: cluster kernel for small vectors, else the persistent cooperative kernel (default);
+    1: three kernels with look-back; 2: the persistent kernel at every size."""
     _check(load().gk_set_path(path))
 
 

@@ -120,7 +120,9 @@ void note_launch(int n = 1);
 // Stage timing: mark(ws, st, i) records event i (0 = before the first kernel) when tracing is on.
 void stage_mark(Workspace* ws, cudaStream_t st, int i);
 int64_t output_capacity(int64_t d);
-int selected_path();  // 0: fused kernel when usable, 1: three kernels with look-back
+int selected_path();  // 0: cluster kernel for small vectors, else the persistent kernel; 1: three kernels; 2: persistent kernel at every size
+int enqueue_gk_small(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
+                     float* val_out, int64_t* nnz_out, cudaStream_t st);
 // eps == nullptr: the operator on a given vector (src = u, read only)
 int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k, int32_t* idx_out,
                      float* val_out, int64_t* nnz_out, cudaStream_t st);

@@ -165,7 +165,7 @@ extern "C" int gk_set_capacity(int64_t cap) {
 }
 
 extern "C" int gk_set_path(int path) {
-    if (path < 0 || path > 1) return GK_ERR_SIZE;
+    if (path < 0 || path > 2) return GK_ERR_SIZE;
     g_path.store(path);
     return GK_OK;
 }

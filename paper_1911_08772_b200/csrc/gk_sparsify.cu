@@ -249,11 +249,16 @@ int enqueue_gk_three_kernel(Workspace* ws, const float* src, float* eps, int64_t
     return GK_OK;
 }
 
-// Enqueue one step by the selected path: the fused cooperative kernel unless it
-// cannot be used on this device (or for this call), else the three-kernel path.
+// Enqueue one step by the selected path: the cluster kernel for small vectors, else the fused
+// cooperative kernel, unless they cannot be used on this device (or for this call), else the
+// three-kernel path.
 // eps == nullptr: the operator form on src = u.
 int enqueue_gk_sparsify(Workspace* ws, const float* src, float* eps, int64_t d, int64_t k,
                         int32_t* idx_out, float* val_out, int64_t* nnz_out, cudaStream_t st) {
+    if (selected_path() == 0) {
+        const int rc = enqueue_gk_small(ws, src, eps, d, k, idx_out, val_out, nnz_out, st);
+        if (rc != 1) return rc;
+    }
     if (selected_path() != 1) {
         const int rc = enqueue_gk_fused(ws, src, eps, d, k, idx_out, val_out, nnz_out, st);
         if (rc != 1) return rc;

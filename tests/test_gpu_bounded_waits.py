@@ -50,6 +50,7 @@ def _raw_call(fn, d, k, g):
 def test_a_grid_barrier_that_cannot_complete_gives_up(d):
     g = wl.normal(d, 1e-3, step=60)
     k = wl.ceil_k(d, 1, 1000)
+    gk.gk_set_path(2)           # the persistent kernel at either size (small vectors go to the cluster kernel otherwise)
     gk.gk_debug_set(gk.KNOB_BARRIER_POLLS, 300)
     gk.gk_debug_set(gk.KNOB_EXTRA_ARRIVALS, 1)
     for _ in range(2):     # twice: the counters are reset by the CTAs that gave up

@@ -26,7 +26,7 @@ def _library():
     gk.gk_set_path(0)
 
 
-@pytest.mark.parametrize("path", [0, 1], ids=["fused", "three_kernel"])
+@pytest.mark.parametrize("path", [0, 1, 2], ids=["default", "three_kernel", "persistent"])
 @pytest.mark.parametrize("max_rounds", [1, 2, 3, 4])
 @pytest.mark.parametrize("unbiased", [True, False])
 def test_rounds_and_divisor(path, max_rounds, unbiased):

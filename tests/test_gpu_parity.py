@@ -26,7 +26,7 @@ def _library():
     yield
 
 
-@pytest.fixture(params=[0, 1], ids=["fused", "three_kernel"])
+@pytest.fixture(params=[0, 1, 2], ids=["default", "three_kernel", "persistent"])
 def gk_path(request):
     """Run a test once per implementation of gk_sparsify."""
     gk.gk_set_path(request.param)
@@ -480,3 +480,25 @@ def test_everything_selected_on_a_vector_of_many_rows(gk_path):
         nn = torch.zeros(4, dtype=torch.int64, device="cuda")
         eps_new, _ = check_segmented_step(step, g, z, offsets, seg_k, dev_off, dev_k, nn)
         assert not eps_new.any()
+
+
+def test_the_three_implementations_agree_on_a_small_vector():
+    # the cluster kernel (default below 589,824 elements), the persistent kernel and the three
+    # kernels: same pairs, same residual, same counts
+    d = 269_722
+    g = wl.normal(d, 1e-3, step=21)
+    e = wl.laplace(d, 1e-3, step=22)
+    step = DeviceStep(d)
+    outs = []
+    for path in (0, 1, 2):
+        gk.gk_set_path(path)
+        try:
+            before = gk.gk_launch_count()
+            eps_new, st = check_gk_step(step, g, e, 270)
+            launches = gk.gk_launch_count() - before
+        finally:
+            gk.gk_set_path(0)
+        assert launches == (3 if path == 1 else 1)
+        outs.append((bits(eps_new).copy(), st.counts, st.nnz, st.rounds))
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0]) and o[1:] == outs[0][1:]

@@ -27,7 +27,7 @@ def _library():
     gk.gk_debug_set(gk.KNOB_PREDICTION, -1)
 
 
-@pytest.fixture(params=[0, 1], ids=["fused", "three_kernel"])
+@pytest.fixture(params=[0, 1, 2], ids=["default", "three_kernel", "persistent"])
 def gk_path(request):
     gk.gk_set_path(request.param)
     yield request.param
