@@ -41,6 +41,8 @@ constexpr int kSmallCells = kSmallMaxRows * kFusedWarps;
 struct __align__(128) SmallShared {
     double2 red[kFusedWarps];
     double2 part;                        // this CTA's sums, read by the others
+    double2 tot;                         // the cluster's sums
+    unsigned int before;                 // survivors in the CTAs before this one
     unsigned int cta_counts[kNumCand];   // this CTA's counts, read by the others
     unsigned int total;                  // this CTA's survivors, read by the others
     unsigned long long col[kNumCand];
@@ -167,13 +169,25 @@ k_gk_small(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
         if (tid == 0) sh.part = part;
         cluster_sync();
-        if (tid == 0) {
-            // the same order in every CTA: identical statistics everywhere
-            double s = 0.0, q = 0.0;
-            for (unsigned int r = 0; r < kSmallCluster; ++r) {
-                s += ld_remote_f64(&sh.part.x, r);
-                q += ld_remote_f64(&sh.part.y, r);
+        if (w == 0) {
+            // lane r fetches CTA r's sums (the loads of all ranks are in flight together); they are
+            // then added in rank order, the same in every CTA: identical statistics everywhere
+            double ps = 0.0, pq = 0.0;
+            if (lane < kSmallCluster) {
+                ps = ld_remote_f64(&sh.part.x, (unsigned int)lane);
+                pq = ld_remote_f64(&sh.part.y, (unsigned int)lane);
             }
+            double s = 0.0, q = 0.0;
+#pragma unroll
+            for (int r = 0; r < kSmallCluster; ++r) {
+                s += __shfl_sync(0xffffffffu, ps, r);
+                q += __shfl_sync(0xffffffffu, pq, r);
+            }
+            if (lane == 0) sh.tot = make_double2(s, q);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const double s = sh.tot.x, q = sh.tot.y;
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
             alg1_thresholds(st, s, q, pv, d, k, z);
             const bool neg = sh.stats.thres0 < 0.0;
@@ -207,10 +221,12 @@ k_gk_small(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
         }
         cluster_sync();
-        if (tid < kNumCand) {
-            unsigned long long s = 0ull;
-            for (unsigned int r = 0; r < kSmallCluster; ++r) s += ld_remote_u32(&sh.cta_counts[tid], r);
-            sh.col[tid] = s;
+        // thread (j, r) fetches CTA r's count of candidate j; sixteen lanes add up one candidate
+        if (tid < kNumCand * kSmallCluster) {
+            unsigned long long v = ld_remote_u32(&sh.cta_counts[tid / kSmallCluster], (unsigned int)(tid % kSmallCluster));
+#pragma unroll
+            for (int o = kSmallCluster / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (tid % kSmallCluster == 0) sh.col[tid / kSmallCluster] = v;
         }
         __syncthreads();
         if (tid == 0) {
@@ -261,8 +277,13 @@ k_gk_small(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         }
         cluster_sync();
         // survivors in the CTAs before this one (the ragged tail comes last of all)
-        unsigned long long before = 0ull;
-        for (unsigned int r = 0; r < c; ++r) before += ld_remote_u32(&sh.total, r);
+        if (w == 0) {
+            const unsigned int t = lane < kSmallCluster ? ld_remote_u32(&sh.total, (unsigned int)lane) : 0u;
+            const unsigned int b = __reduce_add_sync(0xffffffffu, (unsigned int)lane < c ? t : 0u);
+            if (lane == 0) sh.before = b;
+        }
+        __syncthreads();
+        const unsigned long long before = sh.before;
         for (int r = 0; r < nrows; ++r) {
             if (!(all_pass || sh.maxtab[r * kFusedWarps + w] > thr16)) continue;
             const int64_t i = first4 + (int64_t)r * kRowF4;
