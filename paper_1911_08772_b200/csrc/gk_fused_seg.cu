@@ -4,8 +4,10 @@
 //
 // One CTA per SM owns a contiguous run of rows of 1024 float4 (with its own
 // thresholds every segment looks alike to the count phase, so contiguous runs
-// stay balanced, and a run meets only a few segments).  The phases are those of
-// the whole-vector kernel:
+// stay balanced, and a run meets only a few segments).  The runs are cut to
+// equal cost, a segment boundary counting as two rows, so that a stretch of
+// many short layers does not leave one CTA behind.  The phases are those of the
+// whole-vector kernel:
 //
 //   phase A  u = g + eps over eps through the ring of asynchronous copies; the
 //            per-thread fp64 sums belong to the segment the run is in and are
@@ -61,6 +63,7 @@ struct __align__(128) SegFusedShared {
     unsigned int wsum[kFusedWarps];
     unsigned int rowpre[kSfTableMaxRows];              // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kSfGroupRows];
+    int runrow[kFusedGridCap + 1];                     // first row of every CTA's run; [G] = rows of the vector
     unsigned long long total;                          // survivors in the runs before this one
     unsigned int n_staged;                             // survivors whose places were put aside in phase C
     int ok;
@@ -84,12 +87,13 @@ __device__ __forceinline__ int seg_find(const long long* off, int S, int64_t e) 
     return lo;
 }
 
-// rows_per_cta: rows of the run of every CTA; u_slots: row slots of shared memory that hold u
-// after phase A (the last u_slots rows of the run); table_rows = rows_per_cta.
+// n_rows: rows of 1024 float4 in the vector (at least as many as CTAs); max_rows: the most rows a
+// run may have (table entries); u_slots: row slots of shared memory that hold u after phase A
+// (the last u_slots rows of the run).
 // Shared memory: [ring of kSfRing rows][u_slots rows][table of table_rows x 32 uint16].
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, const int64_t* __restrict__ off_g,
-               const int64_t* __restrict__ seg_k, int S, int rows_per_cta, int u_slots, Ctrl* __restrict__ ctrl,
+               const int64_t* __restrict__ seg_k, int S, int n_rows, int max_rows, int u_slots, Ctrl* __restrict__ ctrl,
                SegScratch v, unsigned int* __restrict__ bars, unsigned int* __restrict__ cta_tot,
                int32_t* __restrict__ idx_out, float* __restrict__ val_out, int64_t* __restrict__ seg_nnz_out,
                int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
@@ -102,14 +106,6 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
     const int c = blockIdx.x, G = gridDim.x;
     const int64_t n4 = d >> 2;
 
-    // this CTA's run of float4 and of elements
-    int64_t lo4 = (int64_t)c * rows_per_cta * kRowF4, hi4 = lo4 + (int64_t)rows_per_cta * kRowF4;
-    if (lo4 > n4) lo4 = n4;
-    if (hi4 > n4) hi4 = n4;
-    const int nrows = (int)((hi4 - lo4 + kRowF4 - 1) / kRowF4);
-    const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on stay on chip
-    const int64_t run_lo = lo4 << 2;
-    const int64_t run_hi = (c == G - 1) ? d : (hi4 << 2);           // the last CTA also owns the d mod 4 tail
     const bool owns_tail = (c == G - 1) && (w == kFusedWarps - 1) && (lane < (int)(d & 3));
     const int64_t tail_i = (n4 << 2) + lane;
     const float4* g4 = reinterpret_cast<const float4*>(g);
@@ -127,19 +123,6 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
         if (trace != nullptr && tid == 0) trace[(size_t)c * 8 + slot] = global_timer_ns();
     };
     stamp(0);
-
-    // rows are fetched kSfStages - 1 ahead by asynchronous copies: g into a ring, eps into the slot
-    // that will hold u; the first ones go out before the table is read
-    auto fetch = [&](int r) {
-        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
-        if (r < nrows && i < hi4) {
-            cp_async16(gring + (size_t)(r % kSfStages) * kRowF4 + tid, g4 + i);
-            cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + i);
-        }
-        cp_async_commit();
-    };
-#pragma unroll
-    for (int r = 0; r < kSfStages - 1; ++r) fetch(r);
 
     // ------------------------------------------------------------ the table
     // Offsets and pivots go to shared memory; every CTA checks the table for itself.
@@ -162,7 +145,82 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
     if (c == 0) for (int j = tid; j < S * kNumCand; j += kFusedThreads) v.counts[j] = 0ull;
     __syncthreads();
     const int S_use = bad ? 0 : S;  // a malformed table: u is still formed, nothing is selected
+
+    // ------------------------------------------------------------ the runs
+    // Every CTA owns a contiguous run of rows.  A segment boundary costs a run about as much as
+    // two rows (its sums and counts are closed warp by warp, the next segment's scalars
+    // fetched), and layer tables have stretches of many short segments: runs of equal length
+    // left the CTA with the most boundaries 5 us behind in phase A and 14 us in phase B, with
+    // everyone else waiting at the barriers.  So the runs are cut to equal COST,
+    // cost(row) = row + 2 (boundaries before the row): thread t finds the first row of run t by
+    // bisection; every CTA computes the same cuts.
+    {
+        // With j boundaries before it a row costs row + 2 j, and that holds for the rows from
+        // range_lo(j) to the row that holds boundary j + 1: one bisection over the boundaries finds
+        // the range of a target cost, the row follows by division.
+        const int nbnd = S_use > 0 ? S_use - 1 : 0;                  // boundaries off[1 .. S_use - 1]
+        auto range_lo = [&](const int j) -> long long { return j == 0 ? 0 : sh.off[j] / (4 * kRowF4) + 1; };
+        if (tid <= G) {
+            int cut = tid == G ? n_rows : 0;
+            if (tid > 0 && tid < G) {
+                const long long target = (long long)tid * (1ll * n_rows + 2ll * nbnd) / G;
+                int lo = 0, hi = nbnd;   // last j with 2 range_lo(j) + 3 j <= target
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (range_lo(mid) + 2ll * mid <= target) lo = mid; else hi = mid - 1;
+                }
+                long long row = target - 2ll * lo;
+                if (row < range_lo(lo)) row = range_lo(lo);
+                if (lo < nbnd && row > sh.off[lo + 1] / (4 * kRowF4)) row = sh.off[lo + 1] / (4 * kRowF4) + 1;
+                cut = row < n_rows ? (int)row : n_rows;
+            }
+            sh.runrow[tid] = cut;
+        }
+        __syncthreads();
+        // every run needs a row at least (a single row can hold dozens of boundaries) and none may
+        // have more than the table has entries for.  The cuts usually are like that as they stand;
+        // otherwise one thread moves them apart, and failing that the runs get equal lengths.
+        int good = 1;
+        if (tid < G) {
+            const int len = sh.runrow[tid + 1] - sh.runrow[tid];
+            good = (len >= 1 && len <= max_rows) ? 1 : 0;
+        }
+        good = __syncthreads_and(good);
+        if (!good && tid == 0) {
+            for (int t = 1; t < G; ++t) if (sh.runrow[t] <= sh.runrow[t - 1]) sh.runrow[t] = sh.runrow[t - 1] + 1;
+            for (int t = G - 1; t >= 1; --t) if (sh.runrow[t] >= sh.runrow[t + 1]) sh.runrow[t] = sh.runrow[t + 1] - 1;
+            bool fits = true;
+            for (int t = 0; t < G; ++t) {
+                const int len = sh.runrow[t + 1] - sh.runrow[t];
+                fits = fits && len >= 1 && len <= max_rows;
+            }
+            if (!fits) for (int t = 0; t <= G; ++t) sh.runrow[t] = (int)((long long)t * n_rows / G);
+        }
+        __syncthreads();
+    }
+    // this CTA's run of float4 and of elements
+    int64_t lo4 = (int64_t)sh.runrow[c] * kRowF4, hi4 = (int64_t)sh.runrow[c + 1] * kRowF4;
+    if (lo4 > n4) lo4 = n4;
+    if (hi4 > n4) hi4 = n4;
+    const int nrows = (int)((hi4 - lo4 + kRowF4 - 1) / kRowF4);
+    const int first_kept = nrows > u_slots ? nrows - u_slots : 0;  // rows from here on stay on chip
+    const int64_t run_lo = lo4 << 2;
+    const int64_t run_hi = (c == G - 1) ? d : (hi4 << 2);           // the last CTA also owns the d mod 4 tail
     stamp(1);
+
+    // rows are fetched kSfStages - 1 ahead by asynchronous copies: g into a ring, eps into the slot
+    // that will hold u
+    auto fetch = [&](int r) {
+        const int64_t i = lo4 + (int64_t)r * kRowF4 + tid;
+        if (r < nrows && i < hi4) {
+            cp_async16(gring + (size_t)(r % kSfStages) * kRowF4 + tid, g4 + i);
+            cp_async16(uslot + (size_t)(r % u_slots) * kRowF4 + tid, e4 + i);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int r = 0; r < kSfStages - 1; ++r) fetch(r);
+
 
     // ------------------------------------------------------------------ phase A
     {
@@ -360,10 +418,17 @@ k_gk_fused_seg(const float* __restrict__ g, float* __restrict__ eps, int64_t d, 
             tsel = INFINITY;  // nothing passes
             for (int i = 0; i < kNumCand; ++i) { c32[i] = INFINITY; c64[i] = INFINITY; }
         } else {
-            const int64_t run4 = (int64_t)rows_per_cta * kRowF4;
-            int c0 = (int)((a >> 2) / run4), c1 = (int)(((b - 1) >> 2) / run4);
-            if (c0 > G - 1) c0 = G - 1;
-            if (c1 > G - 1) c1 = G - 1;
+            // the CTAs whose runs hold the segment's first and last element
+            auto cta_of = [&](const long long e) -> int {
+                const long long row = (e >> 2) / kRowF4;
+                int lo = 0, hi = G - 1;   // last t in [0, G - 1] with runrow[t] <= row
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (sh.runrow[mid] <= row) lo = mid; else hi = mid - 1;
+                }
+                return lo;
+            };
+            const int c0 = cta_of(a), c1 = cta_of(b - 1);
             double s1 = 0.0, s2 = 0.0;
             for (int cc = c0; cc <= c1; cc += 8) {
                 double2 p[8];
@@ -947,12 +1012,12 @@ int enqueue_gk_fused_seg(Workspace* ws, const float* g, float* eps, int64_t d, c
     if (!p || !p->usable) return 1;
     const int64_t n4 = d >> 2;
     const int64_t n_rows = (n4 + kRowF4 - 1) / kRowF4;
-    int64_t rows_per_cta = (n_rows + p->grid - 1) / p->grid;
-    if (rows_per_cta < 1) rows_per_cta = 1;
-    if (rows_per_cta > kSfTableMaxRows) return 1;
-    int64_t G = (n_rows + rows_per_cta - 1) / rows_per_cta;
+    int64_t G = n_rows < p->grid ? n_rows : p->grid;
     if (G < 1) G = 1;
-    int rpc = (int)rows_per_cta;
+    // the longest run the kernel's cut can produce: a run's cost is (n_rows + 2 (S - 1)) / G, a row costs 1
+    int64_t max_rows = (n_rows + 2 * (int64_t)(S - 1) + G - 1) / G + 2;
+    if (max_rows > kSfTableMaxRows) return 1;
+    int rpc = (int)max_rows;
     const int64_t left = (int64_t)kSfSmemBudget - (int64_t)kSfRing * kRowBytes - (int64_t)rpc * kSfTableRowBytes;
     int u_slots = (int)(left / kRowBytes);
     if (u_slots > rpc) u_slots = rpc;
@@ -960,6 +1025,7 @@ int enqueue_gk_fused_seg(Workspace* ws, const float* g, float* eps, int64_t d, c
     // copy for a later row would land on the row being read
     if (u_slots < kSfStages && u_slots < rpc) return 1;
     const size_t smem = (size_t)(kSfRing + u_slots) * kRowBytes + (size_t)rpc * kSfTableRowBytes;
+    int n_rows_arg = (int)n_rows;
     int S_arg = (int)S;
     Ctrl* ctrl = ws->ctrl;
     SegScratch v = segmented_views(ws);
@@ -968,10 +1034,10 @@ int enqueue_gk_fused_seg(Workspace* ws, const float* g, float* eps, int64_t d, c
     int64_t cap = output_capacity(d);
     unsigned long long* trace = ws->cta_trace;
     void* args[] = {(void*)&g, (void*)&eps, (void*)&d, (void*)&seg_offsets, (void*)&seg_k, (void*)&S_arg,
-                    (void*)&rpc, (void*)&u_slots, (void*)&ctrl, (void*)&v, (void*)&bars, (void*)&cta_tot,
+                    (void*)&n_rows_arg, (void*)&rpc, (void*)&u_slots, (void*)&ctrl, (void*)&v, (void*)&bars, (void*)&cta_tot,
                     (void*)&idx_out, (void*)&val_out, (void*)&seg_nnz_out, (void*)&nnz_out, (void*)&cap,
                     (void*)&trace};
-    static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused_seg takes 18 arguments");
+    static_assert(sizeof(args) / sizeof(args[0]) == 19, "k_gk_fused_seg takes 19 arguments");
     stage_mark(ws, st, 0);
     GK_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)k_gk_fused_seg, dim3((unsigned)G), dim3(kFusedThreads), args,
                                             smem, st));
