@@ -97,3 +97,15 @@ def test_dgck_argument_validation_happens_on_the_host(lib):
     assert lib.dgck_select(a + 4, 10, 1, a, 5, a, a, a, st) == -4
     assert lib.dgck_sparsify(a, a + 16, 10, 1, a, 5, a, a, a, st) == -5
     assert lib.dgck_sparsify(a, None, 10, 1, a, 5, a, a, a, st) == -1
+
+
+def test_the_operator_and_the_setters_validate_on_the_host(lib):
+    a = 0x1000
+    assert lib.gk_select(None, 10, 1, a, a, a, None) == -1
+    assert lib.gk_select(a, 0, 1, a, a, a, None) == -2
+    assert lib.gk_select(a, 10, 11, a, a, a, None) == -3
+    assert lib.gk_select(a + 4, 10, 1, a, a, a, None) == -4
+    assert lib.gk_set_params(1, 0) == -2 and lib.gk_set_params(0, 5) == -2     # rounds outside 1 .. 4
+    assert lib.gk_set_path(3) == -2 and lib.gk_set_path(-1) == -2
+    assert lib.gk_debug_set(99, 0) == -2 and lib.gk_debug_set(-1, 0) == -2      # unknown keys
+    assert lib.gk_debug_set(0, -2) == -2                                         # value out of range
