@@ -359,7 +359,7 @@ def run_ours(args):
     ms = statistics.median(regions)
     nnz_mean = float(nnz.item())  # of the last step; 12 * nnz is ~0.03 % of the bytes
     # how the last step took its counts: r = 0 when every CTA counted while streaming
-    info = gk.gk_last_path_info() if args.call == "gk" and args.path == 0 else (0, 0, 0, 0, 0)
+    info = gk.gk_last_path_info() if args.call == "gk" and args.path == 0 else (0, 0, 0, 0, 0, 0)
     r_passes = (0.0 if info[4] > 0 and info[1] == info[4] else 1.0) + (1.0 if info[2] else 0.0)
     bytes_step = algorithmic_bytes(d, nnz_mean, r_passes)
     value = whole_job_gbs(world, bytes_step, K, ms)
@@ -655,6 +655,7 @@ def run_ours(args):
             "bytes_model": f"(16 + 4 r) d + 12 nnz, r = {r_passes:g} count passes over u in the last step",
             "counting": {"ctas": info[4], "ctas_with_prediction": info[0], "ctas_whose_bands_held": info[1],
                          "second_full_count": info[2], "cells_left_to_second_phase": info[3],
+                         "ctas_that_counted_a_selection": info[5],
                          "cells": (d // 4096) * 32},
             "timed": f"{len(regions)} repeats of the {K}-step region, median reported "
                      f"(min {min(regions) / K * 1e3:.2f} us, max {max(regions) / K * 1e3:.2f} us per step)",

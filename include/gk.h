@@ -385,18 +385,22 @@ int gk_last_cta_trace(gk_stream_t stream, uint64_t* host_out, int* n_ctas);
  *   key 4  counting against predicted thresholds in the fused gk_sparsify / gk_select
  *          kernel: -1 automatic (large vectors), 0 never, 1 whenever the vector has 128
  *          elements or more
+ *   key 5  the second phase of that kernel counting only the candidates it expects the rounds
+ *          to reach: -1 automatic, 0 never, 1 always and with thres0 alone (any further
+ *          round then asks for a candidate left out, and the count is taken again in full)
  * Returns GK_ERR_SIZE for an unknown key or a value outside [-1, 2^31 - 1].
  */
 int gk_debug_set(int key, int64_t value);
 
 /*
  * How the last single-kernel gk_sparsify / gk_select call on `stream` took its counts
- * (tracing aid).  Synchronises the stream and writes 5 int64 to HOST host_out: CTAs that
+ * (tracing aid).  Synchronises the stream and writes 6 int64 to HOST host_out: CTAs that
  * formed a prediction of the thresholds from the sample; CTAs whose predicted bands held the
  * exact thresholds (their counts come from the first phase plus the cells it left over);
  * 1 if the rounds needed a candidate the short way leaves out, so that a full count followed;
  * (row, warp) cells of 128 elements left to the second phase by CTAs with a prediction; CTAs
- * of the launch (0 if the call did not run that kernel).
+ * of the launch (0 if the call did not run that kernel); CTAs that counted, in the second
+ * phase, only the candidates they expected the rounds to reach.
  */
 int gk_last_path_info(gk_stream_t stream, int64_t* host_out);
 

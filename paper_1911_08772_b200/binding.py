@@ -334,7 +334,7 @@ def gk_last_cta_trace():
     return [tuple(int(buf[i * 8 + j]) for j in range(8)) for i in range(n.value)]
 
 
-KNOB_BARRIER_POLLS, KNOB_LOOKBACK_POLLS, KNOB_EXTRA_ARRIVALS, KNOB_MUTE_TILE, KNOB_PREDICTION = range(5)
+KNOB_BARRIER_POLLS, KNOB_LOOKBACK_POLLS, KNOB_EXTRA_ARRIVALS, KNOB_MUTE_TILE, KNOB_PREDICTION, KNOB_SELECTED_WAY = range(6)
 
 
 def gk_debug_set(key: int, value: int) -> None:
@@ -345,9 +345,9 @@ def gk_debug_set(key: int, value: int) -> None:
 
 def gk_last_path_info():
     """(CTAs with a prediction, CTAs whose bands held, second count needed, cells left to the
-    second phase, CTAs launched) of the last fused gk_sparsify / gk_select call on the current
-    stream.  Synchronises the stream."""
-    out = (C.c_int64 * 5)()
+    second phase, CTAs launched, CTAs that counted a selection of the candidates) of the last
+    fused gk_sparsify / gk_select call on the current stream.  Synchronises the stream."""
+    out = (C.c_int64 * 6)()
     _check(load().gk_last_path_info(_stream(), out))
     return tuple(int(v) for v in out)
 

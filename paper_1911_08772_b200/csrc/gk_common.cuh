@@ -42,9 +42,10 @@ enum Knob {
     kKnobExtraArrivals = 2,   // host: arrivals the fused kernels' barriers expect beyond the grid size
     kKnobMuteTile = 3,        // compaction tile that does not publish its status word (-1: none)
     kKnobPrediction = 4,      // host: -1 automatic, 0 never, 1 whenever possible (gk_fused.cu)
-    kKnobBiasedStd = 5,       // gk_set_params: 1 divides the variance by d instead of d - 1
-    kKnobMaxRounds = 6,       // gk_set_params: rounds of Algorithm 1's loop, 1 .. 4
-    kKnobCount = 7
+    kKnobSelectedWay = 5,     // phase B of the persistent kernel: -1 automatic, 0 never the selected way, 1 thres0 alone selected
+    kKnobBiasedStd = 6,       // gk_set_params: 1 divides the variance by d instead of d - 1
+    kKnobMaxRounds = 7,       // gk_set_params: rounds of Algorithm 1's loop, 1 .. 4
+    kKnobCount = 8
 };
 typedef int (*KnobSetter)(int key, int value);   // returns a cudaError_t as int
 int register_knob_setter(KnobSetter fn);
@@ -80,8 +81,9 @@ struct Ctrl {
     unsigned long long phase_t[8];
     // fused Gaussian_k kernel, how the last call counted: CTAs that formed a prediction, CTAs whose
     // predicted bands held the exact thresholds, whether a second full count was needed, cells
-    // left to phase B by CTAs with a prediction
-    unsigned int path_info[4];
+    // left to phase B by CTAs with a prediction, CTAs that counted only the candidates they
+    // expected the rounds to reach
+    unsigned int path_info[6];
     // gk_error_ratio: ratio, ||u - Comp(u)||^2, ||u||^2
     double diag[4];
     // DGC_k: key of the sampled threshold, candidates at or above it, rank taken in the sample,

@@ -94,6 +94,24 @@ constexpr double kPredSlack = 5e-4;     // added to the relative half width
 constexpr double kPredMaxDelta = 0.05;  // wider bands than this are not worth counting against
 constexpr unsigned int kSparseWay = 2;  // no prediction: the short way is taken when at most 1 cell in 2 is loud
 // candidates that only phase B's full count covers
+// The selected way of phase B: at most kSelMax candidates, those that the rounds can reach
+// according to an estimate of every candidate's count from this CTA's table of cell maxima.
+constexpr int kSelMax = 6;
+constexpr float kSelSigmas = 4.0f;     // width of an estimate's band, in standard errors of the loud-cell count
+constexpr float kSelSlack = 0.10f;     // added to the band: the maxima are rounded, the cells are not a random sample
+constexpr float kSelCluster = 4.0f;    // survivors that sit together in few cells make the estimate too low: upper side only
+constexpr int kSelMinRows = 12;        // rows a CTA must own for its cells to stand for the vector's
+constexpr float kSelFlat = 0.3f;       // loud cells that stay loud at twice the candidate, as a share: above it, no upper side
+constexpr unsigned int kAllCandMask = (1u << kNumCand) - 1u;
+// Test hook: -1 decides by itself, 0 never takes the selected way, 1 takes it with thres0 alone
+// selected (so that any second round finds a candidate left out and the count is taken again).
+static __device__ int g_selected_way = -1;
+static int set_fused_knob(int key, int value) {
+    if (key == kKnobSelectedWay) return (int)cudaMemcpyToSymbol(g_selected_way, &value, sizeof(int));
+    return 0;
+}
+static const int g_fused_knob_registered = register_knob_setter(&set_fused_knob);
+
 constexpr unsigned int kLowCandMask = (1u << cand_index(1, 0)) | (1u << cand_index(2, 0)) |
                                       (1u << cand_index(3, 0)) | (1u << cand_index(2, 1));
 static_assert(cand_by_factor(0) == cand_index(3, 0) && cand_by_factor(1) == cand_index(2, 0) &&
@@ -109,7 +127,7 @@ constexpr int kBarRows = 3;       // barrier inside phase C
 constexpr int kBarInvalid = 14;   // candidates (bit = index) that some CTA has not counted
 constexpr int kBarCounts2 = 15;   // barrier after the second, full count
 constexpr int kBarTotals = 16;    // 2 x kNumCand words: the global counts of the first and the second count
-constexpr int kBarInfo = 36;      // 4 words: what Ctrl::path_info reports, collected during the call
+constexpr int kBarInfo = 36;      // 5 words: what Ctrl::path_info reports, collected during the call
 constexpr int kBarSample = 48;    // 4 doubles: the sample's power sums over all CTAs; then a word: CTAs that are in
 constexpr int kBarWords = 64;
 
@@ -126,7 +144,11 @@ struct __align__(128) FusedShared {
     int ok;
     unsigned int samp_n;                // warps whose sums are in
     int pred_ready;                     // 0: no word yet; 1: the predicted bands stand; 2: no prediction
-    int fast;                           // this CTA's bands hold the exact candidates
+    int fast;                           // phase B of this CTA: 0 in full, 1 a short way over the cells left, 2 the selected way
+    long long k_wanted;                 // k, for the functions that are not handed it
+    int sel_n;                          // the selected way: how many candidates, which (ascending), as a mask
+    int sel_idx[kSelMax];
+    unsigned int sel_mask;
     int recount;                        // the rounds need a candidate that some CTA has not counted
     gk_stats stats;
     unsigned int wsum[kFusedWarps];
@@ -317,22 +339,119 @@ __device__ __forceinline__ Smem smem_of(const int u_slots) {
     (void)gring; (void)uslot; (void)table; (void)lane; (void)w; (void)c; (void)G; (void)nrows; (void)first_kept; \
     (void)n4; (void)stride4; (void)first4; (void)tail_i; (void)in_last_row; (void)owns_tail; (void)sh
 
-// Without a prediction every cell is still to be counted after phase A.  Where few of this
-// CTA's cells can reach even thres0 / 2 (loud layers among quiet ones, heavy tails), the short
-// way over those few -- the six upper candidates and thres0 / 2, which the rounds visit when
-// the first count falls short -- beats streaming every row again; the three lowest candidates
-// then wait for the rounds to ask for them.  Sets sh.fast.  Out of line.
-__device__ __noinline__ void decide_sparse_way(const int64_t d, const int n_rows, const int u_slots) {
+// With every cell still to be counted after phase A, two ways can beat streaming every row
+// against all ten candidates, which is bound by the compare instructions (forty a float4).
+//  - Where few of this CTA's cells can reach even thres0 / 2 (loud layers among quiet ones,
+//    heavy tails), the short way over those few: the six upper candidates and thres0 / 2; the
+//    three lowest candidates then wait for the rounds to ask for them.  sh.fast = 1.
+//  - Else the selected way: the rounds of Algorithm 1 visit four of the ten candidates at most,
+//    and which ones follows from the counts' rough sizes.  The number of cells whose maximum
+//    reaches a candidate gives its count by the Poisson rule (cells without a survivor are
+//    exp(-mean) of all), with a band for the noise of this CTA's cells; a candidate is selected
+//    when the bands leave a way for the rounds to reach it.  Every row is streamed, but only
+//    against the selected candidates.  sh.fast = 2.
+// Either way the candidates left out are flagged, and the rounds asking for one of them sends
+// the CTAs that took a short way through the count in full.  Out of line.
+__device__ __noinline__ void decide_short_way(const int64_t d, const int n_rows, const int u_slots) {
     GK_FUSED_VIEW(d, n_rows, u_slots);
-    if (tid == 0) sh.samp_n = 0u;
+    __syncthreads();   // thread 0 has written the candidates, k and sh.fast
+    const long long k = sh.k_wanted;
+    const int knob = g_selected_way;
+    if (sh.fast != 0 || !(sh.stats.thres0 > 0.0) || nrows == 0) return;   // the same in every thread
+    unsigned int* const wsums = sh.rowpre;   // free until phase C: kNumCand / 2 words per warp
+    // Every warp looks at 32 of its cells at most, evenly spread over its rows: one pass, and a
+    // thousand cells are plenty for the estimate.  (This part and the next are short on work and
+    // long on latency: a lone warp issues an instruction every few cycles.)
+    const int step = (nrows + 31) >> 5;
+    const int looked = (nrows + step - 1) / step;   // rows each warp looks at
+    const unsigned int m = lane < looked ? ((unsigned int)table[lane * step * kFusedWarps + w] & kMaxMask) : 0u;
+    const float n_cells = (float)(looked * kFusedWarps);
+    {
+        // the cells that reach thres0 / 2, counted by the barrier itself
+        const int loud_half = __syncthreads_count(m > (__float_as_uint(sh.cand32[cand_index(1, 0)]) >> 16));
+        if ((float)loud_half * (float)kSparseWay <= n_cells) {
+            if (tid == 0) sh.fast = 1;
+            return;
+        }
+    }
+    if (!(knob > 0 || (knob < 0 && nrows >= kSelMinRows))) return;
+    {
+        // loud cells among them, two candidates to a word
+        unsigned int loud[kNumCand / 2];
+#pragma unroll
+        for (int j = 0; j < kNumCand / 2; ++j) {
+            const unsigned int l0 = __float_as_uint(sh.cand32[2 * j]) >> 16, l1 = __float_as_uint(sh.cand32[2 * j + 1]) >> 16;
+            loud[j] = (m > l0 ? 1u : 0u) + (m > l1 ? 0x10000u : 0u);
+        }
+#pragma unroll
+        for (int j = 0; j < kNumCand / 2; ++j) {
+            const unsigned int ws = __reduce_add_sync(0xffffffffu, loud[j]);
+            if (lane == j) wsums[w * (kNumCand / 2) + j] = ws;
+        }
+    }
     __syncthreads();
-    const unsigned int lim = __float_as_uint(fmaxf(sh.cand32[cand_by_factor(kNumCand - kUpper - 1)], 0.f)) >> 16;
-    unsigned int loud = 0u;
-    for (int rr = lane; rr < nrows; rr += 32) loud += (((unsigned int)table[rr * kFusedWarps + w] & kMaxMask) > lim) ? 1u : 0u;
-    loud = __reduce_add_sync(0xffffffffu, loud);
-    if (lane == 0 && loud) atomicAdd(&sh.samp_n, loud);
-    __syncthreads();
-    if (tid == 0) sh.fast = (sh.stats.thres0 > 0.0 && sh.samp_n * kSparseWay <= (unsigned int)nrows * kFusedWarps) ? 1 : 0;
+    if (w != 0) return;
+    // warp 0: the CTA's sums; then lane j < 10 judges candidate j and ballots carry the judgements
+    float L = 0.f;   // loud cells for this lane's candidate
+#pragma unroll
+    for (int j = 0; j < kNumCand / 2; ++j) {
+        const unsigned int x = __reduce_add_sync(0xffffffffu, wsums[lane * (kNumCand / 2) + j]);
+        if ((lane >> 1) == j) L = (float)((x >> ((lane & 1) * 16)) & 0xffffu);
+    }
+    // Cells that reach a candidate twice as large (the largest there is, for 9/4) in numbers not
+    // far below: loud stretches or lone outliers, not the tail of one bell, and the loud cells
+    // may hold any number of survivors.  No upper side to the estimate then.
+    const int twice = lane == cand_index(0, 0) ? cand_index(0, 2)
+                    : lane == cand_index(1, 0) ? cand_index(0, 0)
+                    : lane == cand_index(0, 1) ? cand_index(0, 3)
+                    : lane == cand_index(2, 0) ? cand_index(1, 0)
+                    : lane == cand_index(1, 1) ? cand_index(0, 1)
+                    : cand_index(0, 3);
+    const float L_twice = __shfl_sync(0xffffffffu, L, twice);
+    bool may_down = false, may_up = false;
+    if (lane < kNumCand) {
+        // the count over the whole vector that this many loud cells among n_cells suggest
+        const float Q = n_cells - L, inv_n = __frcp_rn(n_cells);
+        float lo = 0.f, hi = 5.f * (float)d * (1.f / 128.f) * inv_n * kSelCluster;   // no loud cell: a handful at most
+        if (L > 0.5f) {
+            const float pl = L * inv_n;
+            const float lam = Q < 0.5f ? __logf(2.f * n_cells) : -__logf(1.f - pl);   // survivors per cell
+            const float rel = __fdividef(__fsqrt_rn(pl * inv_n * __frcp_rn(fmaxf(1.f - pl, 0.5f * inv_n))), lam);
+            const float m = 1.f + kSelSigmas * rel + kSelSlack;
+            const float est = lam * (float)d * (1.f / 128.f);
+            lo = __fdividef(est, m);
+            hi = (Q < 8.f || L_twice > kSelFlat * L) ? INFINITY : est * m * kSelCluster;
+        }
+        may_down = 3.f * lo < 2.f * (float)k;
+        may_up = 3.f * hi > 4.f * (float)k;
+    }
+    const unsigned int downs = __ballot_sync(0xffffffffu, may_down), ups = __ballot_sync(0xffffffffu, may_up);
+    // The candidates the rounds can reach: round by round, a step down (to the candidate with one
+    // more halving) where the count may fall short of 2k/3, a step up where it may pass 4k/3.
+    // Lane ci asks whether either of its parents is reached and may step its way.
+    const int b_ = lane < 4 ? 0 : lane < 7 ? 1 : lane < 9 ? 2 : 3;
+    const int h_ = lane - (b_ == 0 ? 0 : b_ == 1 ? 4 : b_ == 2 ? 7 : 9);
+    const int from_above = (lane < kNumCand && h_ > 0) ? cand_index(h_ - 1, b_) : -1;   // reached by a step down
+    const int from_below = (lane < kNumCand && b_ > 0) ? cand_index(h_, b_ - 1) : -1;   // reached by a step up
+    unsigned int reach = 1u << cand_index(0, 0);
+    if (knob != 1) {
+#pragma unroll
+        for (int lvl = 0; lvl < kMaxRounds - 1; ++lvl) {
+            const bool r = (from_above >= 0 && ((reach & downs) >> from_above) & 1u) ||
+                           (from_below >= 0 && ((reach & ups) >> from_below) & 1u);
+            reach |= __ballot_sync(0xffffffffu, r);
+        }
+    }
+    // in ascending order of the thresholds: lane j looks at the j-th smallest candidate
+    int mine_ci = 0;
+#pragma unroll
+    for (int j = 0; j < kNumCand; ++j) if (lane == j) mine_ci = cand_by_factor(j);
+    const bool in = lane < kNumCand && ((reach >> mine_ci) & 1u);
+    const unsigned int sorted = __ballot_sync(0xffffffffu, in);
+    if (__popc(sorted) <= kSelMax) {
+        if (in) sh.sel_idx[__popc(sorted & ((1u << lane) - 1u))] = mine_ci;
+        if (lane == 0) { sh.sel_n = __popc(sorted); sh.sel_mask = reach; sh.fast = 2; }
+    }
 }
 
 // Phase B, the short way: the six upper candidates over the cells that phase A left (flagged),
@@ -440,6 +559,8 @@ __device__ __noinline__ void count_in_full(const float* __restrict__ uvec, const
 #pragma unroll
     for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
     static_assert(kRowF4 == 1024 && (kRing & (kRing - 1)) == 0, "ring indexing assumes 1024-float4 rows, 2^n slots");
+    // (two rows to an iteration: the counting is bound by its compare instructions, and two
+    // independent rows keep the pipes busier than one)
 #pragma unroll 2
     for (int q = 0; q < first_kept; ++q) {
         fetch_u(q + kRing - 1);
@@ -447,6 +568,7 @@ __device__ __noinline__ void count_in_full(const float* __restrict__ uvec, const
         count_float4(gring[((q & (kRing - 1)) << 10) + tid], row_max(first_kept - 1 - q), cs, tier, acc);
     }
     cp_async_wait<0>();
+#pragma unroll 1
     for (int r = first_kept; r < nrows; ++r) {
         if (r != nrows - 1 || in_last_row)
             count_float4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], row_max(r), cs, tier, acc);
@@ -465,6 +587,73 @@ __device__ __noinline__ void count_in_full(const float* __restrict__ uvec, const
     for (int j = 0; j < kNumCand; ++j) {
         const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
         if (lane == 0 && ws) atomicAdd(&sh.cta_counts[sh.order[j]], ws);
+    }
+    __syncthreads();
+}
+
+// Phase B, the selected way: every cell of this CTA against the candidates of sh.sel_idx
+// (ascending; empty places hold +inf, which nothing exceeds).  Every candidate is its own tier:
+// it is evaluated only where the cell's maximum reaches it.
+__device__ __noinline__ void count_selected(const float* __restrict__ uvec, const int64_t d, const int n_rows,
+                                            const int u_slots, const float tail_u) {
+    GK_FUSED_VIEW(d, n_rows, u_slots);
+    const float4* u4 = reinterpret_cast<const float4*>(uvec);
+    const int n_sel = sh.sel_n;
+    float cs[kSelMax], acc[kSelMax];
+    unsigned int lim[kSelMax];
+#pragma unroll
+    for (int j = 0; j < kSelMax; ++j) {
+        cs[j] = j < n_sel ? sh.cand32[sh.sel_idx[j]] : INFINITY;   // all positive: thres0 > 0
+        acc[j] = 0.f;
+        lim[j] = __float_as_uint(cs[j]) >> 16;
+    }
+    const unsigned short* trow = table + w;
+    auto count4 = [&](const float4 v, const unsigned int rm) {   // rm: the cell's maximum, as in count_float4
+        if (rm <= lim[0]) return;
+        const float a0 = fabsf(v.x), a1 = fabsf(v.y), a2 = fabsf(v.z), a3 = fabsf(v.w);
+        count_tier<0, 1>(a0, a1, a2, a3, cs, acc);
+        if (rm <= lim[1]) return;
+        count_tier<1, 2>(a0, a1, a2, a3, cs, acc);
+        if (rm <= lim[2]) return;
+        count_tier<2, 3>(a0, a1, a2, a3, cs, acc);
+        if (rm <= lim[3]) return;
+        count_tier<3, 4>(a0, a1, a2, a3, cs, acc);
+        if (rm <= lim[4]) return;
+        count_tier<4, 5>(a0, a1, a2, a3, cs, acc);
+        if (rm <= lim[5]) return;
+        count_tier<5, 6>(a0, a1, a2, a3, cs, acc);
+    };
+    static_assert(kSelMax == 6, "one tier per selected candidate");
+    // the rows that are not on chip come through the ring, last written first, as in the full count
+    int64_t fo = first4 + (int64_t)(first_kept - 1) * stride4;
+    auto fetch_u = [&](int q) {
+        if (q < first_kept) cp_async16(gring + ((q & (kRing - 1)) << 10) + tid, u4 + fo);
+        cp_async_commit();
+        fo -= stride4;
+    };
+#pragma unroll
+    for (int q = 0; q < kRing - 1; ++q) fetch_u(q);
+#pragma unroll 2
+    for (int q = 0; q < first_kept; ++q) {
+        fetch_u(q + kRing - 1);
+        cp_async_wait<kRing - 1>();
+        count4(gring[((q & (kRing - 1)) << 10) + tid], (unsigned int)trow[(first_kept - 1 - q) * kFusedWarps] & kMaxMask);
+    }
+    cp_async_wait<0>();
+#pragma unroll 1
+    for (int r = first_kept; r < nrows; ++r) {
+        if (r != nrows - 1 || in_last_row)
+            count4(uslot[(size_t)(r % u_slots) * kRowF4 + tid], (unsigned int)trow[r * kFusedWarps] & kMaxMask);
+    }
+    if (owns_tail) {
+        const float a = fabsf(tail_u);
+#pragma unroll
+        for (int j = 0; j < kSelMax; ++j) acc[j] += gt_as_float(a, cs[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < kSelMax; ++j) {
+        const unsigned int ws = __reduce_add_sync(0xffffffffu, (unsigned int)acc[j]);
+        if (lane == 0 && ws && j < n_sel) atomicAdd(&sh.cta_counts[sh.sel_idx[j]], ws);
     }
     __syncthreads();
 }
@@ -511,11 +700,11 @@ __device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, f
                 pending += ql;
             }
             pending = __reduce_add_sync(0xffffffffu, pending);
+            const bool many = pending * 4 > nrows;   // then the rows are taken as they come, eight at a time
             __syncwarp();
             const unsigned int lanes_below = (1u << lane) - 1u;
-            // one segment: x is this thread's float4 of local row r, i its float4 index
-            auto count_cell = [&](const int r, const float4 x, const int64_t i) {
-                const unsigned int m = i < n4 ? mask_above(x, thr) : 0u;
+            // one segment of local row r: m has a bit for each survivor in this thread's float4
+            auto count_cell = [&](const int r, const unsigned int m) {
                 const unsigned int cnt = __reduce_add_sync(0xffffffffu, __popc(m));
                 if (lane == 0) table[r * kFusedWarps + w] = (unsigned short)cnt;
                 if (staged && cnt != 0u) {
@@ -542,48 +731,41 @@ __device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, f
                     }
                 }
             };
-            if (pending * 4 > nrows) {
-                // many qualifying segments: the rows are taken eight at a time as they come
-                for (int r0 = 0; r0 < nrows; r0 += kGroupRows) {
-                    float4 v[kGroupRows];
-                    bool on[kGroupRows];
-#pragma unroll
-                    for (int q = 0; q < kGroupRows; ++q) {
-                        const int r = r0 + q;
-                        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        on[q] = r < nrows && table[r * kFusedWarps + w] == kPending;
-                        if (on[q]) {
-                            const int64_t i = (first4 + (int64_t)r * stride4);
-                            if (i < n4) v[q] = load_row(r, i);
-                        }
-                    }
-#pragma unroll
-                    for (int q = 0; q < kGroupRows; ++q)
-                        if (on[q]) count_cell(r0 + q, v[q], first4 + (int64_t)(r0 + q) * stride4);
-                }
-            } else {
-                // few qualifying segments: they are gathered eight at a time so that their loads overlap
-                for (int cursor = 0; cursor < nrows;) {
-                    const int n = gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w]);
-                    float4 v[kGroupRows];
-#pragma unroll
-                    for (int q = 0; q < kGroupRows; ++q) {
-                        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (q < n) {
-                            const int r = sh.qrow[w][q];
-                            const int64_t i = (first4 + (int64_t)r * stride4);
-                            if (i < n4) v[q] = load_row(r, i);
-                        }
-                    }
-#pragma unroll
-                    for (int q = 0; q < kGroupRows; ++q) {
-                        if (q < n) {
-                            const int r = sh.qrow[w][q];
-                            count_cell(r, v[q], first4 + (int64_t)r * stride4);
-                        }
-                    }
+            // else the qualifying segments are gathered, eight at a time; either way their loads overlap
+            for (int cursor = 0; cursor < nrows;) {
+                int n;
+                if (many) {
+                    n = 0;
+                    const int r = cursor + lane;
+                    const unsigned int pend = __ballot_sync(0xffffffffu, lane < kGroupRows && r < nrows &&
+                                                                             table[r * kFusedWarps + w] == kPending);
+                    if (lane < kGroupRows && ((pend >> lane) & 1u)) sh.qrow[w][__popc(pend & ((1u << lane) - 1u))] = (unsigned short)r;
+                    n = __popc(pend);
+                    cursor += kGroupRows;
                     __syncwarp();
+                } else {
+                    n = gather_cells<kGatherPending>(table, nrows, cursor, sh.qrow[w]);
                 }
+                float4 v[kGroupRows];
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < n) {
+                        const int r = sh.qrow[w][q];
+                        const int64_t i = (first4 + (int64_t)r * stride4);
+                        if (i < n4) v[q] = load_row(r, i);
+                    }
+                }
+                // the eight masks of this thread in one word, so that the segments can be taken one
+                // after the other by one copy of the code
+                unsigned int masks = 0u;
+#pragma unroll
+                for (int q = 0; q < kGroupRows; ++q) {
+                    if (q < n && first4 + (int64_t)sh.qrow[w][q] * stride4 < n4) masks |= mask_above(v[q], thr) << (4 * q);
+                }
+#pragma unroll 1
+                for (int q = 0; q < n; ++q) count_cell(sh.qrow[w][q], (masks >> (4 * q)) & 15u);
+                __syncwarp();
             }
         }
         __syncthreads();
@@ -683,22 +865,25 @@ __device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, f
             // step 3: every warp writes the survivors of its segments that have any
             for (int cursor = 0; cursor < nrows;) {
                 const int n = gather_cells<kGatherNonZero>(table, nrows, cursor, sh.qrow[w]);
-                float4 v[kGroupRows];
+                // (the ring holds no places here: the cells that are not on chip land in it, slot q
+                // for the q-th, and are then taken one after the other)
 #pragma unroll
                 for (int q = 0; q < kGroupRows; ++q) {
-                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (q < n) {
                         const int r = sh.qrow[w][q];
                         const int64_t i = (first4 + (int64_t)r * stride4);
-                        if (i < n4) v[q] = load_row(r, i);
+                        if (i < n4 && r < first_kept) cp_async16(gring + (q << 10) + tid, u4 + i);
                     }
                 }
-#pragma unroll
-                for (int q = 0; q < kGroupRows; ++q) {
-                    if (q >= n) continue;
+                cp_async_commit();
+                cp_async_wait<0>();
+#pragma unroll 1
+                for (int q = 0; q < n; ++q) {
                     const int r = sh.qrow[w][q];
                     const int64_t i = (first4 + (int64_t)r * stride4);
-                    const unsigned int m = i < n4 ? mask_above(v[q], thr) : 0u;
+                    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i < n4) x = (r >= first_kept) ? uslot[(size_t)(r % u_slots) * kRowF4 + tid] : gring[(q << 10) + tid];
+                    const unsigned int m = i < n4 ? mask_above(x, thr) : 0u;
                     // survivors of this row in the warps before this one
                     const unsigned int before =
                         __reduce_add_sync(0xffffffffu, lane < w ? (unsigned int)table[r * kFusedWarps + lane] : 0u);
@@ -712,7 +897,7 @@ __device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, f
                     if (m) {
                         long long p = (long long)sh.rowpre[r] + before + (sc - c_m);
                         const int64_t e0 = i << 2;
-                        const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+                        const float vv[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
                             if (m & (1u << t)) {
@@ -1006,11 +1191,14 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
                 }
             }
             sh.fast = fast ? 1 : 0;
+            sh.k_wanted = k;
             if (PRED && sh.pred_ready == 1) atomicAdd(&bars[kBarInfo + 0], 1u);
             sh.recount = 0;
         }
         if (tid < kNumCand) sh.cta_counts[tid] = 0u;
-        if (!PRED) decide_sparse_way(d, n_rows, u_slots);
+        // (vectors large enough for the prediction are left as they are: where it fails, on heavy
+        // tails or loud stretches, the estimate behind the selected way fails too)
+        if (!PRED) decide_short_way(d, n_rows, u_slots);
         if (c == 0 && tid == 0) ctrl->phase_t[1] = global_timer_ns();
         __syncthreads();
     }
@@ -1020,11 +1208,13 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
     // then ask for a candidate that some CTA left out, the CTAs that took the short way count
     // again in full and the sums are formed a second time.
     for (int pass = 0; pass < 2; ++pass) {
-        const bool fast = pass == 0 && sh.fast != 0;
-        if (fast) {
+        const int way = pass == 0 ? sh.fast : 0;
+        const bool fast = way != 0;
+        if (way == 1) {
             if (PRED) count_short_way<kUpper>(uvec, d, n_rows, u_slots, pacc[0], pacc[1], pacc[2], tail_u, bars);
             else count_short_way<kUpper + 1>(uvec, d, n_rows, u_slots, 0.f, 0.f, 0.f, tail_u, bars);
         }
+        else if (way == 2) count_selected(uvec, d, n_rows, u_slots, tail_u);
         else if (pass == 0 || sh.fast != 0) count_in_full(uvec, d, n_rows, u_slots, tail_u, pass == 1);
         // this CTA's counts join the global sums; the short way leaves the four lower candidates out
         if (tid < kNumCand) {
@@ -1032,8 +1222,9 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
         }
         if (fast && tid == 0) {
-            atomicOr(&bars[kBarInvalid], PRED ? kLowCandMask : (kLowCandMask & ~(1u << cand_index(1, 0))));
-            atomicAdd(&bars[kBarInfo + 1], 1u);
+            atomicOr(&bars[kBarInvalid], way == 2 ? (kAllCandMask & ~sh.sel_mask)
+                                                  : PRED ? kLowCandMask : (kLowCandMask & ~(1u << cand_index(1, 0))));
+            atomicAdd(&bars[kBarInfo + (way == 2 ? 4 : 1)], 1u);
         }
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
         stamp(3);
@@ -1101,7 +1292,7 @@ leave:
             bars[kBarStats] = 0u; bars[kBarCounts] = 0u; bars[kBarRows] = 0u;
             bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
             for (int j = 0; j < 2 * kNumCand; ++j) bars[kBarTotals + j] = 0u;
-            for (int j = 0; j < 4; ++j) { ctrl->path_info[j] = bars[kBarInfo + j]; bars[kBarInfo + j] = 0u; }
+            for (int j = 0; j < 5; ++j) { ctrl->path_info[j] = bars[kBarInfo + j]; bars[kBarInfo + j] = 0u; }
             for (int j = 0; j < 9; ++j) bars[kBarSample + j] = 0u;
             __threadfence();
             bars[kBarExit] = 0u;

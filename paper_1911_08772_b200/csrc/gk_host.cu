@@ -150,7 +150,7 @@ static std::atomic<int> g_host_knob[kKnobCount] = {};
 static std::atomic<bool> g_host_knob_set[kKnobCount] = {};
 int host_knob(int key) {
     if (key < 0 || key >= kKnobCount) return 0;
-    if (!g_host_knob_set[key].load()) return key == kKnobPrediction ? -1 : 0;
+    if (!g_host_knob_set[key].load()) return (key == kKnobPrediction || key == kKnobSelectedWay) ? -1 : 0;
     return g_host_knob[key].load();
 }
 
@@ -246,10 +246,11 @@ extern "C" int gk_last_path_info(gk_stream_t stream, int64_t* host_out) {
     Workspace* ws = find_workspace((cudaStream_t)stream);
     if (!ws) return GK_ERR_NULL;
     GK_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-    unsigned int v[4];
+    unsigned int v[5];
     GK_CUDA_TRY(cudaMemcpy(v, ws->ctrl->path_info, sizeof(v), cudaMemcpyDeviceToHost));
     for (int i = 0; i < 4; ++i) host_out[i] = (int64_t)v[i];
     host_out[4] = ws->last_fused ? ws->last_grid : 0;
+    host_out[5] = (int64_t)v[4];
     return GK_OK;
 }
 
