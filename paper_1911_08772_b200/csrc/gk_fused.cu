@@ -1288,13 +1288,22 @@ leave:
         __threadfence();
         const unsigned int t = atomicAdd(&bars[kBarExit], 1u);
         if (t == (unsigned)G - 1) {
+            // the words to report are read first, all at once: the kernel ends when this thread
+            // does, and a load that waits behind the previous word's stores costs a round trip each
+            unsigned int info[5];
+#pragma unroll
+            for (int j = 0; j < 5; ++j) info[j] = __ldcg(&bars[kBarInfo + j]);
             ctrl->phase_t[6] = global_timer_ns();
             bars[kBarStats] = 0u; bars[kBarCounts] = 0u; bars[kBarRows] = 0u;
             bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
+#pragma unroll
             for (int j = 0; j < 2 * kNumCand; ++j) bars[kBarTotals + j] = 0u;
-            for (int j = 0; j < 5; ++j) { ctrl->path_info[j] = bars[kBarInfo + j]; bars[kBarInfo + j] = 0u; }
+#pragma unroll
             for (int j = 0; j < 9; ++j) bars[kBarSample + j] = 0u;
-            __threadfence();
+#pragma unroll
+            for (int j = 0; j < 5; ++j) { ctrl->path_info[j] = info[j]; bars[kBarInfo + j] = 0u; }
+            // (no fence before the last word: the end of the kernel orders all of these stores
+            // before the next launch on this stream, the only reader)
             bars[kBarExit] = 0u;
         }
     }
