@@ -541,7 +541,8 @@ leave:
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[7] = global_timer_ns();
             bars[0] = 0u;
-            __threadfence();
+            // (no fence: the end of the kernel orders these stores before the next launch on this
+            // stream, the only reader)
             bars[1] = 0u;
         }
     }

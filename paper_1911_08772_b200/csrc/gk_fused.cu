@@ -158,6 +158,7 @@ struct __align__(128) FusedShared {
     unsigned int rowpre[kTableMaxRows];    // survivors in the vector before each row of this CTA
     unsigned short qrow[kFusedWarps][kGroupRows];  // rows a warp has gathered for one batch
     unsigned int n_staged;                 // survivors put aside in phase C
+    unsigned int left_out;                 // candidates (bit = index) that some CTA has not counted
 };
 
 static_assert(offsetof(FusedShared, roundtot) % 16 == 0 && sizeof(unsigned int) * kTableMaxRows >= 64 * kFusedWarps,
@@ -1237,6 +1238,9 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
 
         // -------------------------------------------------------------- the rounds
         if (tid < kNumCand) sh.col[tid] = (unsigned long long)ld_acquire_u32((pass == 0 ? tot0 : tot1) + tid);
+        // (the candidates some CTA left out, fetched beside the counts rather than by thread 0 after
+        // the rounds, where the round trip would be everyone's wait)
+        if (tid == kNumCand) sh.left_out = ld_acquire_u32(&bars[kBarInvalid]);
         __syncthreads();
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
@@ -1244,7 +1248,7 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             sh.chosen = alg1_resolve(st, k, &visited);
             sh.n_staged = 0u;
             // a candidate the rounds evaluated but some CTA did not count: count again, in full
-            sh.recount = (pass == 0 && (visited & ld_acquire_u32(&bars[kBarInvalid])) != 0u) ? 1 : 0;
+            sh.recount = (pass == 0 && (visited & sh.left_out) != 0u) ? 1 : 0;
         }
         __syncthreads();
         if (!sh.recount) break;

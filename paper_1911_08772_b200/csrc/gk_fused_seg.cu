@@ -961,7 +961,8 @@ leave:
         if (t == (unsigned)G - 1) {
             ctrl->phase_t[6] = global_timer_ns();
             bars[0] = 0u; bars[1] = 0u; bars[3] = 0u; bars[4] = 0u;
-            __threadfence();
+            // (no fence: the end of the kernel orders these stores before the next launch on this
+            // stream, the only reader)
             bars[2] = 0u;
         }
     }
