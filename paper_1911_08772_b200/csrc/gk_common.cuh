@@ -98,6 +98,8 @@ struct Workspace {
     int32_t s_cap = 0;
     Ctrl* ctrl = nullptr;
     double2* partials = nullptr;            // kMaxPartials
+    double2* part_recs = nullptr;           // persistent Gaussian_k kernel: one 32-byte record of partial sums per CTA, and one more
+    unsigned int fused_calls = 0;           // launches of that kernel on this workspace (the records carry the number)
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
     unsigned int* cta_counts = nullptr;     // DGC_k and segmented fused kernels: per-CTA words (kFusedGridCap x kNumCand)

@@ -180,6 +180,28 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
     return v;
 }
 
+// A CTA's partial sums travel as one 32-byte record, written with one 256-bit store and read with
+// one 256-bit load: {call number, 0, s, q, 0, call number}.  The record is its own arrival flag:
+// a reader that finds this call's number at both ends has the sums of this call (a 32-byte aligned
+// access is one sector to L2; the number at both ends also shows a record torn between its
+// 16-byte halves, should a device ever do that).  No fence and no counter: the sums are all that
+// the other CTAs need from this one before the second barrier.
+__device__ __forceinline__ void store_partial(unsigned int* rec, const unsigned int call_no, const double s, const double q) {
+    asm volatile("st.relaxed.gpu.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(rec), "r"(call_no), "r"(0u),
+                 "r"((unsigned int)__double2loint(s)), "r"((unsigned int)__double2hiint(s)),
+                 "r"((unsigned int)__double2loint(q)), "r"((unsigned int)__double2hiint(q)), "r"(0u), "r"(call_no)
+                 : "memory");
+}
+__device__ __forceinline__ bool load_partial(const unsigned int* rec, const unsigned int call_no, double& s, double& q) {
+    unsigned int w0, w1, w2, w3, w4, w5, w6, w7;
+    asm volatile("ld.relaxed.gpu.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3), "=r"(w4), "=r"(w5), "=r"(w6), "=r"(w7) : "l"(rec) : "memory");
+    s = __hiloint2double((int)w3, (int)w2);
+    q = __hiloint2double((int)w5, (int)w4);
+    return w0 == call_no && w7 == call_no;
+}
+constexpr int kPartialWords = 8;   // 32 bytes a record
+
 // The predicted first threshold and its bands, from the sample's power sums about the pivot pv
 // (n sample elements).  The half width is kPredSigmas standard errors of mu + sigma z, with the
 // standard error of sigma taken from the sample's own fourth moment (heavy tails widen the
@@ -938,14 +960,15 @@ __device__ __noinline__ bool compact_survivors(const float* __restrict__ uvec, f
 // n_rows: rows of 1024 float4 in the whole vector; CTA c owns rows c, c + G, c + 2G, ...
 // (G = gridDim.x), so that stretches of large values are spread over all CTAs.  u_slots: row
 // slots of shared memory that receive eps and then hold u (the last u_slots rows of a CTA stay
-// on chip); table_rows: the largest number of rows any CTA owns (entries of the maximum table).
+// on chip); call_no: the number of this launch on its scratch, never 0 (the CTAs' records of partial
+// sums carry it; `partials` points to one 32-byte record per CTA and one more).
 // PRED: count during phase A against predicted thresholds (the vector must have at least 32
 // float4 and no CTA more than kPredMaxRows rows); bar_target: arrivals a grid barrier waits for (the grid size; a test may ask for more
 // to see the bounded waits run out).  rowcnt: one word per row.
 template <bool ACC, bool PRED>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, int64_t k, double z,
-           int n_rows, int u_slots, int table_rows, unsigned int bar_target, Ctrl* __restrict__ ctrl,
+           int n_rows, int u_slots, unsigned int call_no, unsigned int bar_target, Ctrl* __restrict__ ctrl,
            double2* __restrict__ partials, unsigned int* __restrict__ bars,
            unsigned int* __restrict__ rowcnt, int32_t* __restrict__ idx_out, float* __restrict__ val_out,
            int64_t* __restrict__ nnz_out, int64_t cap, unsigned long long* __restrict__ trace) {
@@ -954,7 +977,6 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
     float4* e4 = reinterpret_cast<float4*>(eps);
     // where u is read again after phase A: eps holds it for the sparsifier, the input itself otherwise
     const float* uvec = ACC ? eps : src;
-    const float4* u4 = reinterpret_cast<const float4*>(uvec);
     float tail_u = 0.f;
     const bool wide_ok = ACC && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
     unsigned int* tot0 = bars + kBarTotals;               // global counts of the first count
@@ -1161,19 +1183,33 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
             s0 += x; q0 = fma(x, x, q0);
         }
         const double2 part = block_sum2<kFusedThreads>(s0 + s1, q0 + q1, sh.red);
-        if (tid == 0) partials[c] = part;
+        unsigned int* const recs = reinterpret_cast<unsigned int*>(partials);
+        if (tid == 0) store_partial(recs + (size_t)c * kPartialWords, call_no, part.x, part.y);
         stamp(1);
-        if (!grid_barrier(&bars[kBarStats], bar_target, &sh.ok)) {
+        // Grid barrier 1 is the arrival of the sums themselves: thread t waits for the record of
+        // CTA t (bounded polls), and every CTA forms the same totals from the same records in the
+        // same order.  (A counter would cost a fence that waits for this CTA's stores of u, which
+        // nobody else reads, then the counter's round trip, then the records' round trip.)  A
+        // test's extra arrivals are records that nobody writes.
+        double s = 0.0, q = 0.0;
+        bool arrived = true;
+        {
+            const int limit = g_barrier_poll_limit;
+            for (int t = tid; t < (int)bar_target; t += kFusedThreads) {
+                double ps = 0.0, pq = 0.0;
+                int polls = 0;
+                while (!load_partial(recs + (size_t)t * kPartialWords, call_no, ps, pq)) {
+                    if (++polls > limit) { arrived = false; break; }
+                    __nanosleep(100);
+                }
+                if (arrived && t < G) { s += ps; q += pq; }
+            }
+        }
+        if (!__syncthreads_and(arrived)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
         stamp(2);
-        // every CTA forms the same totals: thread t takes partial t, t + T, ...
-        double s = 0.0, q = 0.0;
-        for (int t = tid; t < G; t += kFusedThreads) {
-            const double2 p = __ldcg(&partials[t]);
-            s += p.x; q += p.y;
-        }
         const double2 tot = block_sum2<kFusedThreads>(s, q, sh.red);
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
@@ -1400,16 +1436,17 @@ static bool wants_prediction(const FusedGeometry& geo, int64_t d) {
 // eps == nullptr launches the operator form.
 static cudaError_t launch_fused(const FusedGeometry& geo, cudaStream_t st, const float* src, float* eps, int64_t d,
                                 int64_t k, double z, Ctrl* ctrl, double2* partials, unsigned int* bars, unsigned int* rowcnt, int32_t* idx_out, float* val_out,
-                                int64_t* nnz_out, int64_t cap, unsigned long long* trace) {
-    int n_rows = geo.n_rows, u_slots = geo.u_slots, table_rows = geo.table_rows;
-    unsigned int bar_target = (unsigned int)geo.G + (unsigned int)host_knob(kKnobExtraArrivals);
+                                int64_t* nnz_out, int64_t cap, unsigned long long* trace, unsigned int call_no) {
+    int n_rows = geo.n_rows, u_slots = geo.u_slots;
+    // (a test's extra arrivals: one is as good as many, and the first barrier has one spare record)
+    unsigned int bar_target = (unsigned int)geo.G + (host_knob(kKnobExtraArrivals) > 0 ? 1u : 0u);
     void* args[] = {(void*)&src, (void*)&eps, (void*)&d, (void*)&k, (void*)&z, (void*)&n_rows, (void*)&u_slots,
-                    (void*)&table_rows, (void*)&bar_target, (void*)&ctrl, (void*)&partials,
+                    (void*)&call_no, (void*)&bar_target, (void*)&ctrl, (void*)&partials,
                     (void*)&bars, (void*)&rowcnt, (void*)&idx_out, (void*)&val_out, (void*)&nnz_out, (void*)&cap,
                     (void*)&trace};
     static_assert(sizeof(args) / sizeof(args[0]) == 18, "k_gk_fused takes 18 arguments");
     // the four instances have the same parameter list; naming them keeps the types checked
-    typedef void (*Kern)(const float*, float*, int64_t, int64_t, double, int, int, int, unsigned int, Ctrl*, double2*,
+    typedef void (*Kern)(const float*, float*, int64_t, int64_t, double, int, int, unsigned int, unsigned int, Ctrl*, double2*,
                          unsigned int*, unsigned int*, int32_t*, float*, int64_t*, int64_t, unsigned long long*);
     const bool acc = eps != nullptr, pred = wants_prediction(geo, d);
     const Kern kern = acc ? (pred ? (Kern)k_gk_fused<true, true> : (Kern)k_gk_fused<true, false>)
@@ -1433,7 +1470,8 @@ int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int
     const double z = normal_quantile_upper(1.0 - pq);
     ws->last_grid = (int)geo.G;
     stage_mark(ws, st, 0);
-    GK_CUDA_TRY(launch_fused(geo, st, src, eps, d, k, z, ws->ctrl, ws->partials, ws->bars, ws->rowcnt, idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace));
+    if (++ws->fused_calls == 0u) ws->fused_calls = 1u;   // 0 is what an unwritten record holds
+    GK_CUDA_TRY(launch_fused(geo, st, src, eps, d, k, z, ws->ctrl, ws->part_recs, ws->bars, ws->rowcnt, idx_out, val_out, nnz_out, output_capacity(d), ws->cta_trace, ws->fused_calls));
     note_launch();
     stage_mark(ws, st, 1);
     ws->last_fused = true;
@@ -1460,7 +1498,7 @@ int enqueue_gk_fused(Workspace* ws, const float* src, float* eps, int64_t d, int
 namespace gk {
 
 constexpr size_t kStaticCtrlBytes = (sizeof(Ctrl) + 255) / 256 * 256;
-constexpr size_t kStaticPartialBytes = sizeof(double2) * kFusedGridCap;                // 8 KB
+constexpr size_t kStaticPartialBytes = ((size_t)32 * (kFusedGridCap + 1) + 255) / 256 * 256;   // 16 KB: a 32-byte record per CTA, and one more
 constexpr size_t kStaticBarBytes = sizeof(unsigned int) * kBarWords;          // 256 bytes
 constexpr size_t kStaticHeadBytes = 32 * 1024;             // everything but the per-row words
 constexpr int kStaticRowCap = 1 << 17;                     // rows of 4096 elements: d up to 2^29
@@ -1477,6 +1515,7 @@ struct StaticScratch {
     bool ready = false;
     unsigned char* base = nullptr;
     int sm_count = 0;
+    unsigned int calls = 0;   // launches on this device's array (under g_static_mu)
 };
 static StaticScratch g_static[64];
 static std::mutex g_static_mu;
@@ -1526,8 +1565,14 @@ extern "C" int gk_sparsify_static(const float* g, float* eps, int64_t d, int64_t
     const double pq = 1.0 - (double)k / (double)d;
     const double z = normal_quantile_upper(1.0 - pq);
     unsigned long long* trace = nullptr;  // no trace array in the fixed scratch
+    unsigned int call_no;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (++ss->calls == 0u) ss->calls = 1u;   // 0 is what an unwritten record holds
+        call_no = ss->calls;
+    }
     GK_CUDA_TRY(launch_fused(geo, st, g, eps, d, k, z, ctrl, partials, bars, rowcnt, idx_out, val_out, nnz_out,
-                             output_capacity(d), trace));
+                             output_capacity(d), trace, call_no));
     note_launch();
     return GK_OK;
 }

@@ -49,7 +49,7 @@ int64_t output_capacity(int64_t d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t ctrl, partials, hist, cta_counts, bars, cta_trace, rowcnt, tile_status, seg, total;
+    size_t ctrl, partials, part_recs, hist, cta_counts, bars, cta_trace, rowcnt, tile_status, seg, total;
 };
 
 static Layout layout_for(int64_t d, int32_t S) {
@@ -57,6 +57,7 @@ static Layout layout_for(int64_t d, int32_t S) {
     size_t at = 0;
     L.ctrl = at;        at = align_up(at + sizeof(Ctrl), 256);
     L.partials = at;    at = align_up(at + sizeof(double2) * kMaxPartials, 256);
+    L.part_recs = at;   at = align_up(at + (size_t)32 * (kFusedGridCap + 1), 256);
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
     L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
     L.bars = at;        at = align_up(at + sizeof(unsigned int) * 64, 256);
@@ -98,6 +99,7 @@ int acquire_workspace(int64_t d, int32_t S, cudaStream_t stream, Workspace** out
         ws.s_cap = ns;
         ws.ctrl = reinterpret_cast<Ctrl*>(b + L.ctrl);
         ws.partials = reinterpret_cast<double2*>(b + L.partials);
+        ws.part_recs = reinterpret_cast<double2*>(b + L.part_recs);
         ws.hist = reinterpret_cast<unsigned int*>(b + L.hist);
         ws.cta_counts = reinterpret_cast<unsigned int*>(b + L.cta_counts);
         ws.bars = reinterpret_cast<unsigned int*>(b + L.bars);
