@@ -103,7 +103,7 @@ struct Workspace {
     unsigned long long* tile_status = nullptr;  // one per compaction tile
     unsigned int* hist = nullptr;           // 3 x 2048 radix histograms
     unsigned int* cta_counts = nullptr;     // DGC_k and segmented fused kernels: per-CTA words (kFusedGridCap x kNumCand)
-    unsigned int* bars = nullptr;           // 64 words: [0..3], [9], [14..35] fused sparsifier, [4..8] fused Top_k, [10..13] fused segmented
+    unsigned int* bars = nullptr;           // 128 words: [2..3], [36..56], [64..103] fused sparsifier, [4..8] fused Top_k, [10..13] fused segmented
     unsigned int* rowcnt = nullptr;         // fused kernels: two words per row of 4096 elements
     unsigned long long* cta_trace = nullptr;  // fused kernel: kFusedGridCap x 8 timestamps (tracing aid)
     int last_grid = 0;                      // CTAs of the last fused launch

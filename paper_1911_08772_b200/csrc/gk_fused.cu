@@ -120,16 +120,17 @@ static_assert(cand_by_factor(0) == cand_index(3, 0) && cand_by_factor(1) == cand
 
 // Words of the barrier block used by this kernel (the exact Top_k kernel has 4..8, the segmented
 // one 10..13).  All are zero between calls: the CTA that leaves last clears them.
-constexpr int kBarStats = 0;      // barrier after phase A
-constexpr int kBarCounts = 1;     // barrier after phase B
+// (words 0 and 1 are free: the first two barriers are the arrival of the data itself, see the kernel)
 constexpr int kBarExit = 2;       // CTAs that have left
 constexpr int kBarRows = 3;       // barrier inside phase C
-constexpr int kBarInvalid = 14;   // candidates (bit = index) that some CTA has not counted
-constexpr int kBarCounts2 = 15;   // barrier after the second, full count
-constexpr int kBarTotals = 16;    // 2 x kNumCand words: the global counts of the first and the second count
+constexpr int kBarTotals = 64;    // 2 x kNumCand 64-bit words (first count, second count), one per candidate:
+                                  // CTAs that have added theirs (bits 52..63), CTAs that left the candidate
+                                  // out (40..51), the count over the vector (0..39)
+constexpr int kTotArriveShift = 52, kTotLeftShift = 40;
+constexpr unsigned long long kTotCountMask = (1ull << kTotLeftShift) - 1ull;
 constexpr int kBarInfo = 36;      // 5 words: what Ctrl::path_info reports, collected during the call
 constexpr int kBarSample = 48;    // 4 doubles: the sample's power sums over all CTAs; then a word: CTAs that are in
-constexpr int kBarWords = 64;
+constexpr int kBarWords = 128;
 
 struct __align__(128) FusedShared {
     double2 red[kFusedWarps];
@@ -979,8 +980,8 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
     const float* uvec = ACC ? eps : src;
     float tail_u = 0.f;
     const bool wide_ok = ACC && ((reinterpret_cast<uintptr_t>(eps) & 31u) == 0);  // 32-byte stores possible
-    unsigned int* tot0 = bars + kBarTotals;               // global counts of the first count
-    unsigned int* tot1 = bars + kBarTotals + kNumCand;    // ... of the second, full one
+    unsigned long long* tot0 = reinterpret_cast<unsigned long long*>(bars + kBarTotals);   // first count
+    unsigned long long* tot1 = tot0 + kNumCand;                                            // the second, full one
     if (c == 0 && tid == 0) {
         ctrl->stats.status = GK_DEV_OK;
         ctrl->phase_t[0] = global_timer_ns();
@@ -1253,19 +1254,41 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         }
         else if (way == 2) count_selected(uvec, d, n_rows, u_slots, tail_u);
         else if (pass == 0 || sh.fast != 0) count_in_full(uvec, d, n_rows, u_slots, tail_u, pass == 1);
-        // this CTA's counts join the global sums; the short way leaves the four lower candidates out
+        // Grid barrier 2 is the arrival of the counts themselves.  This CTA's ten counts join ten
+        // 64-bit words, each with a 1 in the word's arrival field and a 1 in its "left out" field
+        // where a short way did not count the candidate; lane j of warp 0 then polls word j until
+        // every CTA has added to it (bounded), and has count, arrivals and left-out flag in one
+        // load: no counter, no fence, no second round trip for the sums.
         if (tid < kNumCand) {
-            const unsigned int v = sh.cta_counts[tid];
-            if (v) atomicAdd((pass == 0 ? tot0 : tot1) + tid, v);
+            const unsigned int left = !fast ? 0u : way == 2 ? (kAllCandMask & ~sh.sel_mask)
+                                                 : PRED ? kLowCandMask : (kLowCandMask & ~(1u << cand_index(1, 0)));
+            atomicAdd((pass == 0 ? tot0 : tot1) + tid,
+                      (1ull << kTotArriveShift) | ((unsigned long long)((left >> tid) & 1u) << kTotLeftShift) |
+                          (unsigned long long)sh.cta_counts[tid]);
         }
-        if (fast && tid == 0) {
-            atomicOr(&bars[kBarInvalid], way == 2 ? (kAllCandMask & ~sh.sel_mask)
-                                                  : PRED ? kLowCandMask : (kLowCandMask & ~(1u << cand_index(1, 0))));
-            atomicAdd(&bars[kBarInfo + (way == 2 ? 4 : 1)], 1u);
-        }
+        if (fast && tid == 0) atomicAdd(&bars[kBarInfo + (way == 2 ? 4 : 1)], 1u);
         if (c == 0 && tid == 0) ctrl->phase_t[2] = global_timer_ns();
         stamp(3);
-        if (!grid_barrier(&bars[pass == 0 ? kBarCounts : kBarCounts2], bar_target, &sh.ok)) {
+        bool arrived = true;
+        if (w == 0) {
+            unsigned long long v = 0ull;
+            if (lane < kNumCand) {
+                const unsigned long long* word = (pass == 0 ? tot0 : tot1) + lane;
+                const int limit = g_barrier_poll_limit;
+                int polls = 0;
+                while (true) {
+                    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
+                    if ((unsigned int)(v >> kTotArriveShift) >= bar_target) break;
+                    if (++polls > limit) { arrived = false; break; }
+                    __nanosleep(40);
+                }
+                sh.col[lane] = v & kTotCountMask;
+            }
+            // the candidates some CTA left out
+            const unsigned int lo = __ballot_sync(0xffffffffu, lane < kNumCand && ((v >> kTotLeftShift) & 0xfffull) != 0ull);
+            if (lane == 0) sh.left_out = lo;
+        }
+        if (!__syncthreads_and(arrived)) {
             if (tid == 0) atomicOr(&ctrl->stats.status, GK_DEV_TIMEOUT);
             goto leave;
         }
@@ -1273,11 +1296,6 @@ k_gk_fused(const float* __restrict__ src, float* __restrict__ eps, int64_t d, in
         stamp(4);
 
         // -------------------------------------------------------------- the rounds
-        if (tid < kNumCand) sh.col[tid] = (unsigned long long)ld_acquire_u32((pass == 0 ? tot0 : tot1) + tid);
-        // (the candidates some CTA left out, fetched beside the counts rather than by thread 0 after
-        // the rounds, where the round trip would be everyone's wait)
-        if (tid == kNumCand) sh.left_out = ld_acquire_u32(&bars[kBarInvalid]);
-        __syncthreads();
         if (tid == 0) {
             const Alg1State st{&sh.stats, sh.cand64, sh.cand32, sh.col, &sh.thr_sel};
             unsigned int visited = 0u;
@@ -1334,10 +1352,9 @@ leave:
 #pragma unroll
             for (int j = 0; j < 5; ++j) info[j] = __ldcg(&bars[kBarInfo + j]);
             ctrl->phase_t[6] = global_timer_ns();
-            bars[kBarStats] = 0u; bars[kBarCounts] = 0u; bars[kBarRows] = 0u;
-            bars[kBarInvalid] = 0u; bars[kBarCounts2] = 0u;
+            bars[kBarRows] = 0u;
 #pragma unroll
-            for (int j = 0; j < 2 * kNumCand; ++j) bars[kBarTotals + j] = 0u;
+            for (int j = 0; j < 2 * kNumCand; ++j) reinterpret_cast<unsigned long long*>(bars + kBarTotals)[j] = 0ull;
 #pragma unroll
             for (int j = 0; j < 9; ++j) bars[kBarSample + j] = 0u;
 #pragma unroll

@@ -60,7 +60,7 @@ static Layout layout_for(int64_t d, int32_t S) {
     L.part_recs = at;   at = align_up(at + (size_t)32 * (kFusedGridCap + 1), 256);
     L.hist = at;        at = align_up(at + sizeof(unsigned int) * 3 * 2048, 256);
     L.cta_counts = at;  at = align_up(at + sizeof(unsigned int) * kFusedGridCap * kNumCand, 256);
-    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 64, 256);
+    L.bars = at;        at = align_up(at + sizeof(unsigned int) * 128, 256);
     L.cta_trace = at;   at = align_up(at + sizeof(unsigned long long) * kFusedGridCap * 8, 256);
     L.rowcnt = at;      at = align_up(at + sizeof(unsigned int) * 2 * ((size_t)(d >> 12) + 2), 256);
     L.tile_status = at; at = align_up(at + sizeof(unsigned long long) * (size_t)num_compact_tiles(d), 256);
